@@ -1,0 +1,194 @@
+/*
+ * cascade.h -- C ABI of the B200 (sm_100a) library for Cascade's sequence-sharded attention.
+ *
+ * The paper (Cascade: Token-Sharded Private LLM Inference) splits the tokens of a layer into disjoint
+ * index sets -- query shards S_j and key/value shards T_k (Section 5.1) -- lets one "AttnNode" per pair
+ * (j, k) compute a partial attention output u with per-row statistics m (row max) and e (sum of
+ * exponentials) (Algorithm 3), and combines the partials over k with a log-sum-exp weighted average
+ * (Section 5.2.3, Algorithm 4 lines 1-8), which reproduces unsharded softmax attention exactly.
+ * This library runs all parties on one GPU.
+ *
+ * Conventions
+ *  - Every function returns a cascade_status_t; CASCADE_OK is 0.  Nothing throws or aborts across the ABI.
+ *    cascade_last_error() returns a thread-local, NUL-terminated description of the last failure.
+ *  - Pointers named *_dev / q / k / v / o_* / m_* / l_* / workspace are DEVICE pointers owned by the
+ *    caller.  Token-to-shard maps and read-back buffers are HOST pointers.
+ *  - All GPU work is enqueued on the caller's stream (a cudaStream_t passed as void*; NULL = default
+ *    stream) without synchronising, except where a function says it synchronises.
+ *  - The library allocates device memory only inside cascade_shard_plan (released by
+ *    cascade_plan_destroy).  Scratch memory is caller-provided after cascade_workspace_bytes.
+ *  - Token ids, shard ids, rows and positions are 0-based.  Query row i of a sequence sits at position
+ *    i + q_pos_offset; KV row y at position y.  With causal != 0 row i sees KV rows y <= i + q_pos_offset.
+ *  - Tensors are token-major: element (b, token, head, c) lives at
+ *    base + b*strides.batch + token*strides.token + head*strides.head + c   (units: elements, c contiguous).
+ *    Row starts must be 16-byte aligned.
+ *  - Query head h reads KV head h / (n_heads / n_kv_heads)  ("repeat_kv", Algorithm 3 lines 1-2).
+ *  - "Shard-major row order": query rows listed shard 0 first, then shard 1, ..., ascending token id
+ *    inside a shard (Section 5.2.2: rows are concatenated in sorted order).  Slot r of that order holds
+ *    token Q_IDX[r].
+ *  - Statistics: m is the true row maximum of the scaled, masked logits in natural-log units, l is
+ *    sum exp(a - m) (the paper's e), both fp32.  A row that sees no key of a shard has m = -inf, l = 0 and
+ *    an all-zero partial output.  The stored partial output is the paper's u: normalised inside its shard.
+ */
+#ifndef CASCADE_H_
+#define CASCADE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t cascade_status_t;
+enum {
+  CASCADE_OK = 0,
+  CASCADE_ERR_INVALID_ARG = 1,  /* null pointer, non-positive size, misaligned pointer or stride */
+  CASCADE_ERR_BAD_MAP = 2,      /* shard id outside [0, n_shards) */
+  CASCADE_ERR_UNSUPPORTED = 3,  /* head_dim not in {64,128}, n_heads % n_kv_heads != 0, unknown dtype */
+  CASCADE_ERR_WORKSPACE = 4,    /* workspace missing or smaller than cascade_workspace_bytes reports */
+  CASCADE_ERR_ALLOC = 5,        /* host or device allocation failed */
+  CASCADE_ERR_CUDA = 6,         /* a CUDA runtime call or launch failed */
+  CASCADE_ERR_TIMEOUT = 7       /* a bounded device-side wait gave up (see cascade_plan_device_status) */
+};
+
+typedef enum { CASCADE_F32 = 0, CASCADE_BF16 = 1 } cascade_dtype_t;
+
+/* Strides in elements; the head_dim axis is contiguous. */
+typedef struct {
+  int64_t batch, token, head;
+} cascade_strides_t;
+
+typedef struct cascade_plan cascade_plan_t; /* opaque, library-owned */
+
+/* Plan arrays readable with cascade_plan_get.  All int32 except PAIR_CLASS (uint8).
+ * Leading dimension n_maps (1 when one map serves the whole batch). */
+enum {
+  CASCADE_PLAN_Q_OFF = 0,      /* [n_maps][n_q_shards+1]   first slot of each query shard            */
+  CASCADE_PLAN_Q_IDX = 1,      /* [n_maps][n_q]            token id held by each shard-major slot     */
+  CASCADE_PLAN_Q_INV = 2,      /* [n_maps][n_q]            slot of each token                         */
+  CASCADE_PLAN_KV_OFF = 3,     /* [n_maps][n_kv_shards+1]                                             */
+  CASCADE_PLAN_KV_IDX = 4,     /* [n_maps][n_kv]                                                      */
+  CASCADE_PLAN_KV_INV = 5,     /* [n_maps][n_kv]                                                      */
+  CASCADE_PLAN_VIS = 6,        /* [n_maps][n_q][n_kv_shards] visible-prefix length of slot r in T_k   */
+  CASCADE_PLAN_PAIR_CLASS = 7  /* [n_maps][n_q_shards][n_kv_shards]  0 EMPTY, 1 PARTIAL, 2 FULL       */
+};
+enum { CASCADE_PAIR_EMPTY = 0, CASCADE_PAIR_PARTIAL = 1, CASCADE_PAIR_FULL = 2 };
+
+int32_t cascade_version(void);
+const char* cascade_last_error(void);
+
+/* Number of kernels this library has launched in this process (monotone; for benchmark accounting). */
+int64_t cascade_launch_count(void);
+
+/*
+ * cascade_shard_plan -- index maps and causal pair mask (Section 5.1 index sets; Section 5.2.2 sorted
+ * concatenation; the sharded mask s^{S_j T_k} = s[:, S_j, T_k]).
+ * Because each shard is kept in ascending token order and the mask is unidirectional, row r of pair
+ * (j, k) sees exactly the first VIS[r][k] keys of T_k (each mask row is visible entries followed by
+ * -inf, Appendix E), so the mask is stored as that prefix length.
+ *   n_maps        1 (one map for every sequence) or the batch size (maps laid out [n_maps][n])
+ *   q_shard_of    HOST int32 [n_maps][n_q],  values in [0, n_q_shards)
+ *   kv_shard_of   HOST int32 [n_maps][n_kv], values in [0, n_kv_shards)
+ *   q_pos_offset  position of query row 0 (0 for prefill, n_kv - n_q for decode with the new tokens
+ *                 already in the cache)
+ *   causal        1 unidirectional mask, 0 no mask
+ * Copies the maps, builds the arrays on the host, uploads them on `stream` and SYNCHRONISES that stream.
+ * Empty shards are allowed.  Errors: INVALID_ARG, BAD_MAP, ALLOC, CUDA.  *out_plan is set only on success.
+ */
+cascade_status_t cascade_shard_plan(int32_t n_maps, int32_t n_q, int32_t n_kv, const int32_t* q_shard_of,
+                                    const int32_t* kv_shard_of, int32_t n_q_shards, int32_t n_kv_shards,
+                                    int32_t q_pos_offset, int32_t causal, void* stream,
+                                    cascade_plan_t** out_plan);
+
+/* Same arrays as cascade_shard_plan, built on the host only: no CUDA call is made, so it works on a machine
+ * without a GPU.  The plan can be read with cascade_plan_get / cascade_plan_dense_mask (device pointers are
+ * NULL) and must be destroyed as usual; the attention calls reject it with INVALID_ARG. */
+cascade_status_t cascade_shard_plan_host(int32_t n_maps, int32_t n_q, int32_t n_kv, const int32_t* q_shard_of,
+                                         const int32_t* kv_shard_of, int32_t n_q_shards, int32_t n_kv_shards,
+                                         int32_t q_pos_offset, int32_t causal, cascade_plan_t** out_plan);
+
+/* Frees host and device memory of a plan (NULL is accepted).  Synchronises the device first. */
+cascade_status_t cascade_plan_destroy(cascade_plan_t* plan);
+
+/* Read-back of a plan array: host copy (library-owned, valid until destroy), device copy and element
+ * count.  Any of the three outputs may be NULL. */
+cascade_status_t cascade_plan_get(const cascade_plan_t* plan, int32_t field, const void** host_ptr,
+                                  const void** dev_ptr, int64_t* n_elems);
+
+/* Dense mask of pair (j, k) of map `map`: host_out[r * |T_k| + c] = 1 if row r of S_j sees key c of T_k.
+ * capacity = bytes available at host_out; WORKSPACE error if smaller than |S_j| * |T_k|. */
+cascade_status_t cascade_plan_dense_mask(const cascade_plan_t* plan, int32_t map, int32_t j, int32_t k,
+                                         uint8_t* host_out, int64_t capacity);
+
+/* Reads the plan's device status word (SYNCHRONISES the device): 0 = no kernel that used this plan hit a
+ * bounded-wait limit; otherwise a code identifying the wait.  Returns TIMEOUT if non-zero. */
+cascade_status_t cascade_plan_device_status(const cascade_plan_t* plan, int32_t* out_code);
+
+/*
+ * cascade_attn_partials -- the attention-pass of every AttnNode_{jk} (Algorithm 3) in one launch:
+ * for each query shard j and KV shard k, a = scale * q^{S_j} (k^{T_k})^T + s^{S_j T_k}; m = row max;
+ * l = row sum exp(a - m); u = softmax(a) v^{T_k}.  Rows of Q/K/V are gathered through the plan's maps.
+ *   q  [batch][n_q][n_heads][head_dim], k, v [batch][n_kv][n_kv_heads][head_dim]  (strides given)
+ *   o_part  [batch][n_kv_shards][n_q shard-major][n_heads][head_dim], same dtype as q, contiguous
+ *   m_part, l_part  fp32 [batch][n_kv_shards][n_q shard-major][n_heads], contiguous
+ * (Together these are the paper's stage-B payload: n_kv_shards * (head_dim + 2) * n_heads * n_q values
+ * per sequence, Appendix D.)  batch must equal n_maps when the plan has per-sequence maps.
+ * head_dim in {64,128}; bf16 with head_dim 128 runs on the tensor cores (tcgen05), everything else on
+ * the fp32 ALU kernel; n_q == 1 with bf16 runs the KV-streaming decode kernel.
+ * workspace: as reported by cascade_workspace_bytes(CASCADE_CALL_PARTIALS) (may be 0 -> NULL allowed).
+ */
+cascade_status_t cascade_attn_partials(const cascade_plan_t* plan, cascade_dtype_t dtype, int32_t batch,
+                                       int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, float scale,
+                                       const void* q, cascade_strides_t q_strides, const void* k,
+                                       cascade_strides_t k_strides, const void* v,
+                                       cascade_strides_t v_strides, void* o_part, float* m_part,
+                                       float* l_part, void* workspace, size_t workspace_bytes,
+                                       void* stream);
+
+/*
+ * cascade_merge -- the post-pass combine (Algorithm 4 lines 1-8; derivation in Section 5.2.3):
+ * n = max_p m_p;  w = sum_p exp(m_p - n) l_p;  o = sum_p exp(m_p - n) l_p u_p / w.
+ * Needs no plan.  Inputs in the layout cascade_attn_partials writes, with n_parts = n_kv_shards.
+ *   row_scatter  DEVICE int32 [n_rows] or NULL: output token row of partial row r (the plan's Q_IDX
+ *                device array); NULL = identity.  With per-sequence maps pass row_scatter_batch_stride
+ *                = n_rows, else 0.
+ *   o_out        [batch][n_rows][n_heads][head_dim] with strides, dtype as the partials
+ *   lse_out      optional fp32 [batch][n_rows][n_heads] (token order): n + ln w; -inf if all parts empty
+ * Rows whose parts are all empty produce zeros.
+ */
+cascade_status_t cascade_merge(cascade_dtype_t dtype, int32_t batch, int32_t n_parts, int32_t n_rows,
+                               int32_t n_heads, int32_t head_dim, const void* o_part, const float* m_part,
+                               const float* l_part, const int32_t* row_scatter,
+                               int64_t row_scatter_batch_stride, void* o_out, cascade_strides_t o_strides,
+                               float* lse_out, void* stream);
+
+/*
+ * cascade_attn_sharded -- attention-pass and post-pass fused (Algorithm 3 followed by Algorithm 4 lines
+ * 1-8): walks the KV shards of the plan one after another for each query-shard tile and carries
+ * (n, w, o) across shards, so no partial is written to memory; by the identity of Section 5.2.3 the
+ * result equals cascade_merge(cascade_attn_partials(...)).  Output in token order:
+ *   o_out [batch][n_q][n_heads][head_dim] with strides; lse_out optional fp32 [batch][n_q][n_heads].
+ * For n_q == 1 (decode, Appendix F "Caching") the KV shards are processed as independent partials in
+ * `workspace` and merged by a second launch.
+ */
+cascade_status_t cascade_attn_sharded(const cascade_plan_t* plan, cascade_dtype_t dtype, int32_t batch,
+                                      int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, float scale,
+                                      const void* q, cascade_strides_t q_strides, const void* k,
+                                      cascade_strides_t k_strides, const void* v,
+                                      cascade_strides_t v_strides, void* o_out,
+                                      cascade_strides_t o_strides, float* lse_out, void* workspace,
+                                      size_t workspace_bytes, void* stream);
+
+enum { CASCADE_CALL_PARTIALS = 0, CASCADE_CALL_SHARDED = 1 };
+
+/* Scratch bytes the given call needs for this plan and shape (0 if none).  The workspace must be
+ * 256-byte aligned. */
+cascade_status_t cascade_workspace_bytes(const cascade_plan_t* plan, int32_t which_call,
+                                         cascade_dtype_t dtype, int32_t batch, int32_t n_heads,
+                                         int32_t n_kv_heads, int32_t head_dim, size_t* out_bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CASCADE_H_ */

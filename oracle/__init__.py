@@ -127,9 +127,10 @@ def dense_mask(plan: Plan, j: int, k: int) -> np.ndarray:
     return (cols[None, :] <= rows[:, None]).astype(np.uint8)
 
 
-def attn_pass(q, k, v, scale, plan: Plan):
+def attn_pass(q, k, v, scale, plan: Plan, row_tokens=None):
     """Per-(query shard, KV shard) partials, Algorithm 3.  Returns (u, m, e) in fp64 with
-    u [B, n_kv_shards, n_q, H, d] and m, e [B, n_kv_shards, n_q, H]; rows in shard-major slot order."""
+    u [B, n_kv_shards, n_rows, H, d] and m, e [B, n_kv_shards, n_rows, H]; rows are the query tokens listed in
+    ``row_tokens`` (default: every slot in shard-major order, plan.q_idx)."""
     lib = _load()
     q, qp = _f32(q)
     k, kp = _f32(k)
@@ -138,13 +139,16 @@ def attn_pass(q, k, v, scale, plan: Plan):
     _, n_kv, Hkv, _ = k.shape
     assert n_q == plan.n_q and n_kv == plan.n_kv
     P = plan.n_kv_shards
-    u = np.empty((B, P, n_q, H, d), np.float64)
-    m = np.empty((B, P, n_q, H), np.float64)
-    e = np.empty((B, P, n_q, H), np.float64)
+    rows, rows_p = _i32(plan.q_idx if row_tokens is None else row_tokens)
+    n_rows = rows.shape[0]
+    u = np.empty((B, P, n_rows, H, d), np.float64)
+    m = np.empty((B, P, n_rows, H), np.float64)
+    e = np.empty((B, P, n_rows, H), np.float64)
     lib.oracle_attn_pass(
         ctypes.c_int(B), ctypes.c_int(n_q), ctypes.c_int(n_kv), ctypes.c_int(H), ctypes.c_int(Hkv),
         ctypes.c_int(d), ctypes.c_double(scale), ctypes.c_int(plan.q_pos_offset),
-        ctypes.c_int(int(plan.causal)), qp, kp, vp, _ptr(plan.q_idx), ctypes.c_int(P), _ptr(plan.kv_off),
+        ctypes.c_int(int(plan.causal)), qp, kp, vp, rows_p, ctypes.c_int(n_rows), ctypes.c_int(P),
+        _ptr(plan.kv_off),
         _ptr(plan.kv_idx), _ptr(u), _ptr(m), _ptr(e))
     return u, m, e
 

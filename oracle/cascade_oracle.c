@@ -183,31 +183,32 @@ int oracle_shard_plan(int n_q, int n_kv, const int32_t* q_shard_of, const int32_
  * step by step as printed:   a = scale * q k^T + s ;  m = row_max(a) ;  a = exp(a - m) ;
  * e = row_sum(a) ;  a = a / e ;  u = a v.
  * The mask s is 0 where KV position <= query position and -inf elsewhere (all 0 if !causal).
- * Row order of the outputs is shard-major query slots (q_idx order):
- *   u[B][n_kv_shards][n_q][H][d],  m,e[B][n_kv_shards][n_q][H]   (double).
+ * Rows evaluated: the n_rows query tokens listed in row_tok (normally q_idx, i.e. every slot in shard-major
+ * order; a subset is allowed so that large cases can be sampled).  Outputs:
+ *   u[B][n_kv_shards][n_rows][H][d],  m,e[B][n_kv_shards][n_rows][H]   (double).
  * A row that sees no key of the shard has m = -inf, e = 0, u = 0 (the printed steps would divide by
  * zero there; the post-pass gives such a term weight zero).
  */
 void oracle_attn_pass(int B, int n_q, int n_kv, int H, int Hkv, int d, double scale,
                       int q_pos_offset, int causal, const float* q, const float* k, const float* v,
-                      const int32_t* q_idx, int n_kv_shards, const int32_t* kv_off,
+                      const int32_t* row_tok, int n_rows, int n_kv_shards, const int32_t* kv_off,
                       const int32_t* kv_idx, double* u, double* m, double* e) {
-  const long total = (long)B * n_kv_shards * n_q * H;
+  const long total = (long)B * n_kv_shards * n_rows * H;
 #pragma omp parallel
   {
     double* a = (double*)malloc(sizeof(double) * (size_t)(n_kv > 0 ? n_kv : 1));
 #pragma omp for schedule(dynamic, 16)
     for (long job = 0; job < total; ++job) {
       const int h = (int)(job % H);
-      const int r = (int)((job / H) % n_q);
-      const int kk = (int)((job / ((long)H * n_q)) % n_kv_shards);
-      const int b = (int)(job / ((long)H * n_q * n_kv_shards));
+      const int r = (int)((job / H) % n_rows);
+      const int kk = (int)((job / ((long)H * n_rows)) % n_kv_shards);
+      const int b = (int)(job / ((long)H * n_rows * n_kv_shards));
       const int g = kv_head_of(h, H, Hkv);
-      const int tok = q_idx[r];
+      const int tok = row_tok[r];
       const long pos = (long)tok + q_pos_offset;
       const float* qr = q + (((size_t)b * n_q + tok) * H + h) * d;
       const int lo = kv_off[kk], hi = kv_off[kk + 1], len = hi - lo;
-      const size_t stat = (((size_t)b * n_kv_shards + kk) * n_q + r) * H + h;
+      const size_t stat = (((size_t)b * n_kv_shards + kk) * n_rows + r) * H + h;
       double* urow = u + stat * d;
       for (int c = 0; c < d; ++c) urow[c] = 0.0;
       /* line 3: masked logits of this row against the whole shard */

@@ -1,0 +1,262 @@
+"""ctypes binding of libcascade_b200.so: argument marshalling only -- every step runs in the CUDA library.
+
+Function names match the C ABI (include/cascade.h).  torch supplies device memory and the current stream.
+The library must have been built (``python -m paper_2507_05228_b200.build``); loading fails loudly otherwise:
+there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcascade_b200.so")
+
+F32, BF16 = 0, 1
+CALL_PARTIALS, CALL_SHARDED = 0, 1
+PLAN_FIELDS = {"q_off": 0, "q_idx": 1, "q_inv": 2, "kv_off": 3, "kv_idx": 4, "kv_inv": 5, "vis": 6,
+               "pair_class": 7}
+STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_MAP", 3: "UNSUPPORTED", 4: "WORKSPACE", 5: "ALLOC", 6: "CUDA",
+                7: "TIMEOUT"}
+
+EXPORTS = [
+    "cascade_version", "cascade_last_error", "cascade_launch_count", "cascade_shard_plan", "cascade_shard_plan_host",
+    "cascade_plan_destroy",
+    "cascade_plan_get", "cascade_plan_dense_mask", "cascade_plan_device_status", "cascade_attn_partials",
+    "cascade_merge", "cascade_attn_sharded", "cascade_workspace_bytes",
+]
+
+
+class CascadeError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"cascade status {status} ({STATUS_NAMES.get(status, '?')}): {message}")
+        self.status = status
+
+
+class Strides(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int64), ("token", ctypes.c_int64), ("head", ctypes.c_int64)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2507_05228_b200.build` "
+                "(there is no CPU or PyTorch fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float
+        L.cascade_version.restype = i32
+        L.cascade_last_error.restype = ctypes.c_char_p
+        L.cascade_launch_count.restype = i64
+        L.cascade_shard_plan.argtypes = [i32, i32, i32, vp, vp, i32, i32, i32, i32, vp, ctypes.POINTER(vp)]
+        L.cascade_shard_plan_host.argtypes = [i32, i32, i32, vp, vp, i32, i32, i32, i32, ctypes.POINTER(vp)]
+        L.cascade_plan_destroy.argtypes = [vp]
+        L.cascade_plan_get.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(i64)]
+        L.cascade_plan_dense_mask.argtypes = [vp, i32, i32, i32, vp, i64]
+        L.cascade_plan_device_status.argtypes = [vp, ctypes.POINTER(i32)]
+        L.cascade_attn_partials.argtypes = [vp, i32, i32, i32, i32, i32, f32, vp, Strides, vp, Strides, vp, Strides,
+                                            vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.cascade_merge.argtypes = [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, i64, vp, Strides, vp, vp]
+        L.cascade_attn_sharded.argtypes = [vp, i32, i32, i32, i32, i32, f32, vp, Strides, vp, Strides, vp, Strides,
+                                           vp, Strides, vp, vp, ctypes.c_size_t, vp]
+        L.cascade_workspace_bytes.argtypes = [vp, i32, i32, i32, i32, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
+        for name in EXPORTS:
+            if name not in ("cascade_version", "cascade_last_error", "cascade_launch_count"):
+                getattr(L, name).restype = i32
+        _lib = L
+    return _lib
+
+
+def _check(status: int):
+    if status != 0:
+        raise CascadeError(status, lib().cascade_last_error().decode())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise CascadeError(3, f"dtype {t.dtype} unsupported")
+
+
+def _strides(t: torch.Tensor) -> Strides:
+    assert t.dim() == 4 and t.stride(3) == 1, "expected [batch, tokens, heads, head_dim] with contiguous head_dim"
+    return Strides(t.stride(0), t.stride(1), t.stride(2))
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream if torch.cuda.is_available() else 0
+
+
+def cascade_version() -> int:
+    return int(lib().cascade_version())
+
+
+def cascade_launch_count() -> int:
+    return int(lib().cascade_launch_count())
+
+
+class Plan:
+    """Owner of a cascade_plan_t*."""
+
+    def __init__(self, handle: int, n_maps: int, n_q: int, n_kv: int, n_q_shards: int, n_kv_shards: int):
+        self.handle = handle
+        self.n_maps, self.n_q, self.n_kv = n_maps, n_q, n_kv
+        self.n_q_shards, self.n_kv_shards = n_q_shards, n_kv_shards
+
+    def get(self, field: str) -> np.ndarray:
+        """Host copy of a plan array (cascade_plan_get)."""
+        hp, n = ctypes.c_void_p(), ctypes.c_int64()
+        _check(lib().cascade_plan_get(self.handle, PLAN_FIELDS[field], ctypes.byref(hp), None, ctypes.byref(n)))
+        ctype = ctypes.c_uint8 if field == "pair_class" else ctypes.c_int32
+        arr = np.ctypeslib.as_array(ctypes.cast(hp, ctypes.POINTER(ctype)), shape=(n.value,)).copy()
+        return arr.reshape(self._shape(field))
+
+    def dev_ptr(self, field: str) -> int:
+        dp = ctypes.c_void_p()
+        _check(lib().cascade_plan_get(self.handle, PLAN_FIELDS[field], None, ctypes.byref(dp), None))
+        return dp.value
+
+    def _shape(self, field):
+        m = self.n_maps
+        return {"q_off": (m, self.n_q_shards + 1), "kv_off": (m, self.n_kv_shards + 1), "q_idx": (m, self.n_q),
+                "q_inv": (m, self.n_q), "kv_idx": (m, self.n_kv), "kv_inv": (m, self.n_kv),
+                "vis": (m, self.n_q, self.n_kv_shards),
+                "pair_class": (m, self.n_q_shards, self.n_kv_shards)}[field]
+
+    def dense_mask(self, j: int, k: int, map: int = 0) -> np.ndarray:
+        qo, ko = self.get("q_off")[map], self.get("kv_off")[map]
+        rows, cols = int(qo[j + 1] - qo[j]), int(ko[k + 1] - ko[k])
+        out = np.zeros((rows, cols), np.uint8)
+        _check(lib().cascade_plan_dense_mask(self.handle, map, j, k, out.ctypes.data_as(ctypes.c_void_p),
+                                             out.size))
+        return out
+
+    def device_status(self) -> int:
+        code = ctypes.c_int32()
+        _check(lib().cascade_plan_device_status(self.handle, ctypes.byref(code)))
+        return code.value
+
+    def destroy(self):
+        if self.handle:
+            lib().cascade_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def _maps(q_shard_of, kv_shard_of):
+    qs = np.ascontiguousarray(q_shard_of, dtype=np.int32)
+    ks = np.ascontiguousarray(kv_shard_of, dtype=np.int32)
+    if qs.ndim == 1:
+        qs, ks = qs[None], ks[None]
+    assert ks.shape[0] == qs.shape[0]
+    return qs, ks
+
+
+def cascade_shard_plan(q_shard_of, kv_shard_of, n_q_shards: int, n_kv_shards: int, q_pos_offset: int = 0,
+                       causal: bool = True) -> Plan:
+    """q_shard_of / kv_shard_of: int32 host arrays [n] (one map for the batch) or [n_maps, n]."""
+    qs, ks = _maps(q_shard_of, kv_shard_of)
+    n_maps, n_q = qs.shape
+    n_kv = ks.shape[1]
+    out = ctypes.c_void_p()
+    _check(lib().cascade_shard_plan(n_maps, n_q, n_kv, qs.ctypes.data_as(ctypes.c_void_p),
+                                    ks.ctypes.data_as(ctypes.c_void_p), n_q_shards, n_kv_shards, q_pos_offset,
+                                    int(bool(causal)), _stream(), ctypes.byref(out)))
+    return Plan(out.value, n_maps, n_q, n_kv, n_q_shards, n_kv_shards)
+
+
+def cascade_shard_plan_host(q_shard_of, kv_shard_of, n_q_shards: int, n_kv_shards: int, q_pos_offset: int = 0,
+                            causal: bool = True) -> Plan:
+    """Host-only plan (no GPU needed): readable, not usable by the attention calls."""
+    qs, ks = _maps(q_shard_of, kv_shard_of)
+    n_maps, n_q = qs.shape
+    n_kv = ks.shape[1]
+    out = ctypes.c_void_p()
+    _check(lib().cascade_shard_plan_host(n_maps, n_q, n_kv, qs.ctypes.data_as(ctypes.c_void_p),
+                                         ks.ctypes.data_as(ctypes.c_void_p), n_q_shards, n_kv_shards, q_pos_offset,
+                                         int(bool(causal)), ctypes.byref(out)))
+    return Plan(out.value, n_maps, n_q, n_kv, n_q_shards, n_kv_shards)
+
+
+def cascade_workspace_bytes(plan: Plan, which_call: int, dtype_code: int, batch: int, n_heads: int, n_kv_heads: int,
+                            head_dim: int) -> int:
+    out = ctypes.c_size_t()
+    _check(lib().cascade_workspace_bytes(plan.handle, which_call, dtype_code, batch, n_heads, n_kv_heads, head_dim,
+                                         ctypes.byref(out)))
+    return out.value
+
+
+def _ws(nbytes: int, device, workspace: Optional[torch.Tensor]):
+    if nbytes == 0:
+        return None, 0, 0
+    if workspace is None:
+        workspace = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    return workspace, workspace.data_ptr(), workspace.numel() * workspace.element_size()
+
+
+def cascade_attn_partials(plan: Plan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, scale: float, out=None,
+                          workspace=None):
+    """Returns (o_part [B, n_kv_shards, n_q, H, d] in q.dtype, m_part, l_part [B, n_kv_shards, n_q, H] fp32);
+    rows in shard-major order."""
+    B, n_q, H, d = q.shape
+    Hkv = k.shape[2]
+    code = _dtype_code(q)
+    if out is None:
+        P = plan.n_kv_shards
+        out = (torch.empty((B, P, n_q, H, d), dtype=q.dtype, device=q.device),
+               torch.empty((B, P, n_q, H), dtype=torch.float32, device=q.device),
+               torch.empty((B, P, n_q, H), dtype=torch.float32, device=q.device))
+    o_part, m_part, l_part = out
+    nbytes = cascade_workspace_bytes(plan, CALL_PARTIALS, code, B, H, Hkv, d)
+    ws, ws_ptr, ws_bytes = _ws(nbytes, q.device, workspace)
+    _check(lib().cascade_attn_partials(plan.handle, code, B, H, Hkv, d, scale, q.data_ptr(), _strides(q),
+                                       k.data_ptr(), _strides(k), v.data_ptr(), _strides(v), o_part.data_ptr(),
+                                       m_part.data_ptr(), l_part.data_ptr(), ws_ptr, ws_bytes, _stream()))
+    return o_part, m_part, l_part
+
+
+def cascade_merge(o_part: torch.Tensor, m_part: torch.Tensor, l_part: torch.Tensor, row_scatter_ptr: int = 0,
+                  row_scatter_batch_stride: int = 0, out=None, want_lse: bool = True):
+    """o_part [B, P, n_rows, H, d]; row_scatter_ptr: device pointer of an int32 [n_rows] map (a plan's q_idx) or 0.
+    Returns (o [B, n_rows, H, d], lse [B, n_rows, H] or None)."""
+    B, P, n_rows, H, d = o_part.shape
+    code = _dtype_code(o_part)
+    o = out if out is not None else torch.empty((B, n_rows, H, d), dtype=o_part.dtype, device=o_part.device)
+    lse = torch.empty((B, n_rows, H), dtype=torch.float32, device=o_part.device) if want_lse else None
+    _check(lib().cascade_merge(code, B, P, n_rows, H, d, o_part.data_ptr(), m_part.data_ptr(), l_part.data_ptr(),
+                               row_scatter_ptr or None, row_scatter_batch_stride, o.data_ptr(), _strides(o),
+                               lse.data_ptr() if lse is not None else None, _stream()))
+    return o, lse
+
+
+def cascade_attn_sharded(plan: Plan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, scale: float, out=None,
+                         want_lse: bool = True, workspace=None):
+    """Fused attention-pass + post-pass.  Returns (o [B, n_q, H, d] in token order, lse or None)."""
+    B, n_q, H, d = q.shape
+    Hkv = k.shape[2]
+    code = _dtype_code(q)
+    o = out if out is not None else torch.empty((B, n_q, H, d), dtype=q.dtype, device=q.device)
+    lse = torch.empty((B, n_q, H), dtype=torch.float32, device=q.device) if want_lse else None
+    nbytes = cascade_workspace_bytes(plan, CALL_SHARDED, code, B, H, Hkv, d)
+    ws, ws_ptr, ws_bytes = _ws(nbytes, q.device, workspace)
+    _check(lib().cascade_attn_sharded(plan.handle, code, B, H, Hkv, d, scale, q.data_ptr(), _strides(q),
+                                      k.data_ptr(), _strides(k), v.data_ptr(), _strides(v), o.data_ptr(),
+                                      _strides(o), lse.data_ptr() if lse is not None else None, ws_ptr, ws_bytes,
+                                      _stream()))
+    return o, lse

@@ -1,0 +1,603 @@
+// C ABI entry points: argument checks, plan construction (host) and kernel dispatch.
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <atomic>
+#include <new>
+
+#include "cascade_internal.cuh"
+
+namespace cascade {
+
+static thread_local char g_err[512] = "";
+static std::atomic<int64_t> g_launches{0};
+
+void set_error(const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+}
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static cascade_status_t cuda_fail(cudaError_t e, const char* what) {
+  set_error("%s: %s", what, cudaGetErrorString(e));
+  return CASCADE_ERR_CUDA;
+}
+
+// Query tiles of `rows_per_tile` slots that stay inside one shard, heaviest first.
+static void build_qtiles(const cascade_plan& pl, int map, int rows_per_tile, std::vector<int4>& out) {
+  struct Tile {
+    int4 t;
+    int64_t work;
+  };
+  std::vector<Tile> tiles;
+  const int nq = pl.dev.n_q, P = pl.dev.n_kv_shards, J = pl.dev.n_q_shards;
+  const int32_t* off = pl.q_off.data() + (size_t)map * (J + 1);
+  const int32_t* vis = pl.vis.data() + (size_t)map * nq * P;
+  for (int j = 0; j < J; ++j) {
+    for (int r0 = off[j]; r0 < off[j + 1]; r0 += rows_per_tile) {
+      const int n = std::min(rows_per_tile, off[j + 1] - r0);
+      int64_t work = 0;
+      for (int k = 0; k < P; ++k) work += vis[(size_t)(r0 + n - 1) * P + k];
+      tiles.push_back({make_int4(r0, n, j, 0), work});
+    }
+  }
+  std::stable_sort(tiles.begin(), tiles.end(), [](const Tile& a, const Tile& b) { return a.work > b.work; });
+  out.clear();
+  for (auto& t : tiles) out.push_back(t.t);
+}
+
+}  // namespace cascade
+
+using namespace cascade;
+
+extern "C" {
+
+int32_t cascade_version(void) { return 100; }
+const char* cascade_last_error(void) { return g_err; }
+int64_t cascade_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+static cascade_status_t plan_host(int32_t n_maps, int32_t n_q, int32_t n_kv, const int32_t* q_shard_of,
+                                  const int32_t* kv_shard_of, int32_t n_q_shards, int32_t n_kv_shards,
+                                  int32_t q_pos_offset, int32_t causal, cascade_plan_t** out_plan) {
+  if (!out_plan || !q_shard_of || !kv_shard_of) {
+    set_error("cascade_shard_plan: null pointer");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (n_maps < 1 || n_q < 1 || n_kv < 1 || n_q_shards < 1 || n_kv_shards < 1) {
+    set_error("cascade_shard_plan: sizes must be positive (n_maps=%d n_q=%d n_kv=%d shards=%d/%d)", n_maps,
+              n_q, n_kv, n_q_shards, n_kv_shards);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  for (int64_t i = 0; i < (int64_t)n_maps * n_q; ++i)
+    if (q_shard_of[i] < 0 || q_shard_of[i] >= n_q_shards) {
+      set_error("cascade_shard_plan: q_shard_of[%lld] = %d outside [0,%d)", (long long)i, q_shard_of[i],
+                n_q_shards);
+      return CASCADE_ERR_BAD_MAP;
+    }
+  for (int64_t i = 0; i < (int64_t)n_maps * n_kv; ++i)
+    if (kv_shard_of[i] < 0 || kv_shard_of[i] >= n_kv_shards) {
+      set_error("cascade_shard_plan: kv_shard_of[%lld] = %d outside [0,%d)", (long long)i, kv_shard_of[i],
+                n_kv_shards);
+      return CASCADE_ERR_BAD_MAP;
+    }
+  cascade_plan* pl = new (std::nothrow) cascade_plan();
+  if (!pl) {
+    set_error("cascade_shard_plan: host allocation failed");
+    return CASCADE_ERR_ALLOC;
+  }
+  try {
+    const int J = n_q_shards, P = n_kv_shards;
+    memset(&pl->dev, 0, sizeof(pl->dev));
+    pl->dev.n_maps = n_maps;
+    pl->dev.n_q = n_q;
+    pl->dev.n_kv = n_kv;
+    pl->dev.n_q_shards = J;
+    pl->dev.n_kv_shards = P;
+    pl->dev.q_pos_offset = q_pos_offset;
+    pl->dev.causal = causal ? 1 : 0;
+    pl->q_off.assign((size_t)n_maps * (J + 1), 0);
+    pl->kv_off.assign((size_t)n_maps * (P + 1), 0);
+    pl->q_idx.assign((size_t)n_maps * n_q, 0);
+    pl->q_inv.assign((size_t)n_maps * n_q, 0);
+    pl->kv_idx.assign((size_t)n_maps * n_kv, 0);
+    pl->kv_inv.assign((size_t)n_maps * n_kv, 0);
+    pl->vis.assign((size_t)n_maps * n_q * P, 0);
+    pl->pair_class.assign((size_t)n_maps * J * P, 0);
+    int max_len = 0;
+    // counting sort of token ids by shard id: ascending ids inside every shard
+    auto sort_by_shard = [](const int32_t* shard_of, int n, int S, int32_t* off, int32_t* idx, int32_t* inv) {
+      std::vector<int32_t> cursor(S + 1, 0);
+      for (int t = 0; t < n; ++t) cursor[shard_of[t] + 1]++;
+      for (int s = 0; s < S; ++s) cursor[s + 1] += cursor[s];
+      for (int s = 0; s <= S; ++s) off[s] = cursor[s];
+      for (int t = 0; t < n; ++t) {
+        const int slot = cursor[shard_of[t]]++;
+        idx[slot] = t;
+        inv[t] = slot;
+      }
+    };
+    for (int mp = 0; mp < n_maps; ++mp) {
+      int32_t* qo = pl->q_off.data() + (size_t)mp * (J + 1);
+      int32_t* ko = pl->kv_off.data() + (size_t)mp * (P + 1);
+      int32_t* qi = pl->q_idx.data() + (size_t)mp * n_q;
+      int32_t* ki = pl->kv_idx.data() + (size_t)mp * n_kv;
+      sort_by_shard(q_shard_of + (size_t)mp * n_q, n_q, J, qo, qi, pl->q_inv.data() + (size_t)mp * n_q);
+      sort_by_shard(kv_shard_of + (size_t)mp * n_kv, n_kv, P, ko, ki, pl->kv_inv.data() + (size_t)mp * n_kv);
+      int32_t* vis = pl->vis.data() + (size_t)mp * n_q * P;
+      for (int k = 0; k < P; ++k) {
+        const int32_t* tb = ki + ko[k];
+        const int32_t* te = ki + ko[k + 1];
+        max_len = std::max(max_len, (int)(te - tb));
+        for (int r = 0; r < n_q; ++r) {
+          int32_t c;
+          if (!causal) {
+            c = (int32_t)(te - tb);
+          } else {
+            const int64_t pos = (int64_t)qi[r] + q_pos_offset;
+            if (pos < 0) c = 0;
+            else if (pos >= n_kv) c = (int32_t)(te - tb);
+            else c = (int32_t)(std::upper_bound(tb, te, (int32_t)pos) - tb);
+          }
+          vis[(size_t)r * P + k] = c;
+        }
+      }
+      uint8_t* pc = pl->pair_class.data() + (size_t)mp * J * P;
+      for (int j = 0; j < J; ++j)
+        for (int k = 0; k < P; ++k) {
+          const int len = ko[k + 1] - ko[k];
+          uint8_t cls = CASCADE_PAIR_EMPTY;
+          if (qo[j + 1] > qo[j] && len > 0) {
+            // rows ascend in position, so the first row has the shortest prefix and the last the longest
+            const int lo = vis[(size_t)qo[j] * P + k], hi = vis[(size_t)(qo[j + 1] - 1) * P + k];
+            if (hi == 0) cls = CASCADE_PAIR_EMPTY;
+            else if (lo == len) cls = CASCADE_PAIR_FULL;
+            else cls = CASCADE_PAIR_PARTIAL;
+          }
+          pc[(size_t)j * P + k] = cls;
+        }
+    }
+    pl->dev.max_kv_shard_len = max_len;
+    // tile lists, padded to the same length for every map
+    std::vector<std::vector<int4>> t32(n_maps), t128(n_maps);
+    size_t n32 = 0, n128 = 0;
+    for (int mp = 0; mp < n_maps; ++mp) {
+      build_qtiles(*pl, mp, 32, t32[mp]);
+      build_qtiles(*pl, mp, 128, t128[mp]);
+      n32 = std::max(n32, t32[mp].size());
+      n128 = std::max(n128, t128[mp].size());
+    }
+    pl->qtiles32.assign(n32 * n_maps, make_int4(0, 0, 0, 0));
+    pl->qtiles128.assign(n128 * n_maps, make_int4(0, 0, 0, 0));
+    for (int mp = 0; mp < n_maps; ++mp) {
+      std::copy(t32[mp].begin(), t32[mp].end(), pl->qtiles32.begin() + mp * n32);
+      std::copy(t128[mp].begin(), t128[mp].end(), pl->qtiles128.begin() + mp * n128);
+    }
+    pl->dev.n_qtiles32 = (int32_t)n32;
+    pl->dev.n_qtiles128 = (int32_t)n128;
+  } catch (const std::bad_alloc&) {
+    delete pl;
+    set_error("cascade_shard_plan: host allocation failed");
+    return CASCADE_ERR_ALLOC;
+  }
+  *out_plan = pl;
+  return CASCADE_OK;
+}
+
+cascade_status_t cascade_shard_plan_host(int32_t n_maps, int32_t n_q, int32_t n_kv, const int32_t* q_shard_of,
+                                         const int32_t* kv_shard_of, int32_t n_q_shards, int32_t n_kv_shards,
+                                         int32_t q_pos_offset, int32_t causal, cascade_plan_t** out_plan) {
+  return plan_host(n_maps, n_q, n_kv, q_shard_of, kv_shard_of, n_q_shards, n_kv_shards, q_pos_offset, causal,
+                   out_plan);
+}
+
+cascade_status_t cascade_shard_plan(int32_t n_maps, int32_t n_q, int32_t n_kv, const int32_t* q_shard_of,
+                                    const int32_t* kv_shard_of, int32_t n_q_shards, int32_t n_kv_shards,
+                                    int32_t q_pos_offset, int32_t causal, void* stream,
+                                    cascade_plan_t** out_plan) {
+  cascade_plan* pl = nullptr;
+  cascade_status_t hs = plan_host(n_maps, n_q, n_kv, q_shard_of, kv_shard_of, n_q_shards, n_kv_shards,
+                                  q_pos_offset, causal, &pl);
+  if (hs != CASCADE_OK) return hs;
+  *out_plan = nullptr;
+
+  // one device blob, every array 256-byte aligned
+  struct Seg {
+    const void* src;
+    size_t bytes;
+    size_t off;
+  };
+  Seg segs[] = {
+      {pl->q_off.data(), pl->q_off.size() * 4, 0},       {pl->q_idx.data(), pl->q_idx.size() * 4, 0},
+      {pl->q_inv.data(), pl->q_inv.size() * 4, 0},       {pl->kv_off.data(), pl->kv_off.size() * 4, 0},
+      {pl->kv_idx.data(), pl->kv_idx.size() * 4, 0},     {pl->kv_inv.data(), pl->kv_inv.size() * 4, 0},
+      {pl->vis.data(), pl->vis.size() * 4, 0},           {pl->pair_class.data(), pl->pair_class.size(), 0},
+      {pl->qtiles32.data(), pl->qtiles32.size() * 16, 0}, {pl->qtiles128.data(), pl->qtiles128.size() * 16, 0},
+  };
+  size_t total = 256;  // status word first
+  for (auto& s : segs) {
+    s.off = total;
+    total += align_up(s.bytes, 256);
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = cudaMalloc(&pl->dev_blob, total);
+  if (e != cudaSuccess) {
+    delete pl;
+    set_error("cascade_shard_plan: cudaMalloc(%zu): %s", total, cudaGetErrorString(e));
+    return CASCADE_ERR_ALLOC;
+  }
+  pl->dev_blob_bytes = total;
+  char* base = (char*)pl->dev_blob;
+  e = cudaMemsetAsync(base, 0, 256, st);
+  for (auto& s : segs)
+    if (e == cudaSuccess && s.bytes) e = cudaMemcpyAsync(base + s.off, s.src, s.bytes, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) {
+    cudaFree(pl->dev_blob);
+    delete pl;
+    return cuda_fail(e, "cascade_shard_plan: upload");
+  }
+  pl->dev.status = (int32_t*)base;
+  pl->dev.q_off = (const int32_t*)(base + segs[0].off);
+  pl->dev.q_idx = (const int32_t*)(base + segs[1].off);
+  pl->dev.q_inv = (const int32_t*)(base + segs[2].off);
+  pl->dev.kv_off = (const int32_t*)(base + segs[3].off);
+  pl->dev.kv_idx = (const int32_t*)(base + segs[4].off);
+  pl->dev.kv_inv = (const int32_t*)(base + segs[5].off);
+  pl->dev.vis = (const int32_t*)(base + segs[6].off);
+  pl->dev.pair_class = (const uint8_t*)(base + segs[7].off);
+  pl->dev.qtiles32 = (const int4*)(base + segs[8].off);
+  pl->dev.qtiles128 = (const int4*)(base + segs[9].off);
+  *out_plan = pl;
+  return CASCADE_OK;
+}
+
+cascade_status_t cascade_plan_destroy(cascade_plan_t* plan) {
+  if (!plan) return CASCADE_OK;
+  if (!plan->dev_blob) {  // host-only plan: nothing on the device
+    delete plan;
+    return CASCADE_OK;
+  }
+  cudaError_t e = cudaDeviceSynchronize();
+  cudaFree(plan->dev_blob);
+  delete plan;
+  if (e != cudaSuccess) return cuda_fail(e, "cascade_plan_destroy: device synchronize");
+  return CASCADE_OK;
+}
+
+cascade_status_t cascade_plan_get(const cascade_plan_t* plan, int32_t field, const void** host_ptr,
+                                  const void** dev_ptr, int64_t* n_elems) {
+  if (!plan) {
+    set_error("cascade_plan_get: null plan");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  const void* h = nullptr;
+  const void* d = nullptr;
+  int64_t n = 0;
+  switch (field) {
+    case CASCADE_PLAN_Q_OFF: h = plan->q_off.data(); d = plan->dev.q_off; n = plan->q_off.size(); break;
+    case CASCADE_PLAN_Q_IDX: h = plan->q_idx.data(); d = plan->dev.q_idx; n = plan->q_idx.size(); break;
+    case CASCADE_PLAN_Q_INV: h = plan->q_inv.data(); d = plan->dev.q_inv; n = plan->q_inv.size(); break;
+    case CASCADE_PLAN_KV_OFF: h = plan->kv_off.data(); d = plan->dev.kv_off; n = plan->kv_off.size(); break;
+    case CASCADE_PLAN_KV_IDX: h = plan->kv_idx.data(); d = plan->dev.kv_idx; n = plan->kv_idx.size(); break;
+    case CASCADE_PLAN_KV_INV: h = plan->kv_inv.data(); d = plan->dev.kv_inv; n = plan->kv_inv.size(); break;
+    case CASCADE_PLAN_VIS: h = plan->vis.data(); d = plan->dev.vis; n = plan->vis.size(); break;
+    case CASCADE_PLAN_PAIR_CLASS:
+      h = plan->pair_class.data(); d = plan->dev.pair_class; n = plan->pair_class.size(); break;
+    default:
+      set_error("cascade_plan_get: unknown field %d", field);
+      return CASCADE_ERR_INVALID_ARG;
+  }
+  if (host_ptr) *host_ptr = h;
+  if (dev_ptr) *dev_ptr = d;
+  if (n_elems) *n_elems = n;
+  return CASCADE_OK;
+}
+
+cascade_status_t cascade_plan_dense_mask(const cascade_plan_t* plan, int32_t map, int32_t j, int32_t k,
+                                         uint8_t* host_out, int64_t capacity) {
+  if (!plan || !host_out) {
+    set_error("cascade_plan_dense_mask: null pointer");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  const PlanDev& d = plan->dev;
+  if (map < 0 || map >= d.n_maps || j < 0 || j >= d.n_q_shards || k < 0 || k >= d.n_kv_shards) {
+    set_error("cascade_plan_dense_mask: index out of range");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  const int32_t* qo = plan->q_off.data() + (size_t)map * (d.n_q_shards + 1);
+  const int32_t* ko = plan->kv_off.data() + (size_t)map * (d.n_kv_shards + 1);
+  const int rows = qo[j + 1] - qo[j], cols = ko[k + 1] - ko[k];
+  if ((int64_t)rows * cols > capacity) {
+    set_error("cascade_plan_dense_mask: need %lld bytes, have %lld", (long long)rows * cols, (long long)capacity);
+    return CASCADE_ERR_WORKSPACE;
+  }
+  const int32_t* vis = plan->vis.data() + (size_t)map * d.n_q * d.n_kv_shards;
+  for (int r = 0; r < rows; ++r) {
+    const int c_vis = vis[(size_t)(qo[j] + r) * d.n_kv_shards + k];
+    for (int c = 0; c < cols; ++c) host_out[(size_t)r * cols + c] = c < c_vis ? 1 : 0;
+  }
+  return CASCADE_OK;
+}
+
+cascade_status_t cascade_plan_device_status(const cascade_plan_t* plan, int32_t* out_code) {
+  if (!plan || !out_code || !plan->dev_blob) {
+    set_error("cascade_plan_device_status: null pointer or host-only plan");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemcpy(out_code, plan->dev.status, 4, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e, "cascade_plan_device_status");
+  if (*out_code != 0) {
+    set_error("device status word = %d: a bounded wait inside a kernel gave up", *out_code);
+    return CASCADE_ERR_TIMEOUT;
+  }
+  return CASCADE_OK;
+}
+
+}  // extern "C"
+
+namespace cascade {
+
+static size_t elt_size(cascade_dtype_t t) { return t == CASCADE_BF16 ? 2 : 4; }
+
+static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+static bool strides_ok(const cascade_strides_t& s, size_t es) {
+  return (s.batch * (int64_t)es) % 16 == 0 && (s.token * (int64_t)es) % 16 == 0 && (s.head * (int64_t)es) % 16 == 0;
+}
+
+static cascade_status_t check_attn_args(const char* fn, const cascade_plan_t* plan, cascade_dtype_t dtype,
+                                        int32_t batch, int32_t H, int32_t Hkv, int32_t d, const void* q,
+                                        const cascade_strides_t& qs, const void* k, const cascade_strides_t& ks,
+                                        const void* v, const cascade_strides_t& vs) {
+  if (!plan || !q || !k || !v) {
+    set_error("%s: null pointer", fn);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (!plan->dev_blob) {
+    set_error("%s: the plan was built by cascade_shard_plan_host and has no device arrays", fn);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (dtype != CASCADE_F32 && dtype != CASCADE_BF16) {
+    set_error("%s: unknown dtype %d", fn, (int)dtype);
+    return CASCADE_ERR_UNSUPPORTED;
+  }
+  if (batch < 1 || H < 1 || Hkv < 1) {
+    set_error("%s: batch and head counts must be positive", fn);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (H % Hkv != 0) {
+    set_error("%s: n_heads %d is not a multiple of n_kv_heads %d", fn, H, Hkv);
+    return CASCADE_ERR_UNSUPPORTED;
+  }
+  if (d != 64 && d != 128) {
+    set_error("%s: head_dim %d unsupported (64 or 128)", fn, d);
+    return CASCADE_ERR_UNSUPPORTED;
+  }
+  if (plan->dev.n_maps != 1 && plan->dev.n_maps != batch) {
+    set_error("%s: plan has %d maps but batch is %d", fn, plan->dev.n_maps, batch);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  const size_t es = elt_size(dtype);
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !strides_ok(qs, es) || !strides_ok(ks, es) ||
+      !strides_ok(vs, es)) {
+    set_error("%s: q/k/v pointers and row strides must be 16-byte aligned", fn);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if ((int64_t)batch * std::max(plan->dev.n_kv_shards, 1) > 65535) {
+    set_error("%s: batch * n_kv_shards exceeds 65535", fn);
+    return CASCADE_ERR_UNSUPPORTED;
+  }
+  return CASCADE_OK;
+}
+
+static AttnParams make_params(const cascade_plan_t* plan, int32_t batch, int32_t H, int32_t Hkv, int32_t d,
+                              float scale, const void* q, const cascade_strides_t& qs, const void* k,
+                              const cascade_strides_t& ks, const void* v, const cascade_strides_t& vs) {
+  AttnParams p;
+  memset(&p, 0, sizeof(p));
+  p.plan = plan->dev;
+  p.q = q;
+  p.k = k;
+  p.v = v;
+  p.qs = {qs.batch, qs.token, qs.head};
+  p.ks = {ks.batch, ks.token, ks.head};
+  p.vs = {vs.batch, vs.token, vs.head};
+  p.batch = batch;
+  p.H = H;
+  p.Hkv = Hkv;
+  p.G = H / Hkv;
+  p.d = d;
+  p.scale = scale;
+  return p;
+}
+
+static bool use_decode(const cascade_plan_t* plan, cascade_dtype_t dtype, int H, int Hkv, int d) {
+  const int G = H / Hkv;
+  return plan->dev.n_q == 1 && dtype == CASCADE_BF16 && d == 128 && (G == 1 || G == 2 || G == 4 || G == 8);
+}
+static bool use_tc(const cascade_plan_t* plan, cascade_dtype_t dtype, int d) {
+  return false && dtype == CASCADE_BF16 && d == 128 && plan->dev.n_q > 1;
+}
+
+static size_t decode_ws_bytes(const cascade_plan_t* plan, cascade_dtype_t dtype, int batch, int H, int d) {
+  const size_t rows = (size_t)batch * plan->dev.n_kv_shards * plan->dev.n_q * H;
+  return align_up(rows * d * elt_size(dtype), 256) + 2 * align_up(rows * 4, 256);
+}
+
+}  // namespace cascade
+
+extern "C" {
+
+cascade_status_t cascade_workspace_bytes(const cascade_plan_t* plan, int32_t which_call, cascade_dtype_t dtype,
+                                         int32_t batch, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim,
+                                         size_t* out_bytes) {
+  if (!plan || !out_bytes) {
+    set_error("cascade_workspace_bytes: null pointer");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (batch < 1 || n_heads < 1 || n_kv_heads < 1 || n_heads % n_kv_heads != 0) {
+    set_error("cascade_workspace_bytes: bad batch or head counts");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (which_call == CASCADE_CALL_PARTIALS) {
+    *out_bytes = 0;
+  } else if (which_call == CASCADE_CALL_SHARDED) {
+    *out_bytes = use_decode(plan, dtype, n_heads, n_kv_heads, head_dim)
+                     ? decode_ws_bytes(plan, dtype, batch, n_heads, head_dim)
+                     : 0;
+  } else {
+    set_error("cascade_workspace_bytes: unknown call %d", which_call);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  return CASCADE_OK;
+}
+
+cascade_status_t cascade_attn_partials(const cascade_plan_t* plan, cascade_dtype_t dtype, int32_t batch,
+                                       int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, float scale,
+                                       const void* q, cascade_strides_t q_strides, const void* k,
+                                       cascade_strides_t k_strides, const void* v, cascade_strides_t v_strides,
+                                       void* o_part, float* m_part, float* l_part, void* workspace,
+                                       size_t workspace_bytes, void* stream) {
+  (void)workspace;
+  (void)workspace_bytes;
+  cascade_status_t s = check_attn_args("cascade_attn_partials", plan, dtype, batch, n_heads, n_kv_heads,
+                                       head_dim, q, q_strides, k, k_strides, v, v_strides);
+  if (s != CASCADE_OK) return s;
+  if (!o_part || !m_part || !l_part) {
+    set_error("cascade_attn_partials: null output pointer");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (!aligned16(o_part) || !aligned16(m_part) || !aligned16(l_part)) {
+    set_error("cascade_attn_partials: outputs must be 16-byte aligned");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  AttnParams p = make_params(plan, batch, n_heads, n_kv_heads, head_dim, scale, q, q_strides, k, k_strides, v,
+                             v_strides);
+  p.fused = 0;
+  p.o_part = o_part;
+  p.m_part = m_part;
+  p.l_part = l_part;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e;
+  if (use_decode(plan, dtype, n_heads, n_kv_heads, head_dim)) e = launch_decode(p, st);
+  else if (use_tc(plan, dtype, head_dim)) e = launch_attn_tc(p, st);
+  else e = launch_attn_simt(p, dtype, st);
+  if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_partials: launch");
+  return CASCADE_OK;
+}
+
+cascade_status_t cascade_merge(cascade_dtype_t dtype, int32_t batch, int32_t n_parts, int32_t n_rows,
+                               int32_t n_heads, int32_t head_dim, const void* o_part, const float* m_part,
+                               const float* l_part, const int32_t* row_scatter, int64_t row_scatter_batch_stride,
+                               void* o_out, cascade_strides_t o_strides, float* lse_out, void* stream) {
+  if (!o_part || !m_part || !l_part || !o_out) {
+    set_error("cascade_merge: null pointer");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (dtype != CASCADE_F32 && dtype != CASCADE_BF16) {
+    set_error("cascade_merge: unknown dtype %d", (int)dtype);
+    return CASCADE_ERR_UNSUPPORTED;
+  }
+  if (batch < 1 || n_parts < 1 || n_rows < 1 || n_heads < 1) {
+    set_error("cascade_merge: sizes must be positive");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (head_dim != 64 && head_dim != 128) {
+    set_error("cascade_merge: head_dim %d unsupported (64 or 128)", head_dim);
+    return CASCADE_ERR_UNSUPPORTED;
+  }
+  if (!aligned16(o_part) || !aligned16(o_out) || !strides_ok(o_strides, elt_size(dtype))) {
+    set_error("cascade_merge: partial/output pointers and row strides must be 16-byte aligned");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  MergeParams p;
+  p.o_part = o_part;
+  p.m_part = m_part;
+  p.l_part = l_part;
+  p.row_scatter = row_scatter;
+  p.row_scatter_batch_stride = row_scatter_batch_stride;
+  p.o_out = o_out;
+  p.os = {o_strides.batch, o_strides.token, o_strides.head};
+  p.lse_out = lse_out;
+  p.batch = batch;
+  p.n_parts = n_parts;
+  p.n_rows = n_rows;
+  p.H = n_heads;
+  p.d = head_dim;
+  cudaError_t e = launch_merge(p, dtype, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e, "cascade_merge: launch");
+  return CASCADE_OK;
+}
+
+cascade_status_t cascade_attn_sharded(const cascade_plan_t* plan, cascade_dtype_t dtype, int32_t batch,
+                                      int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, float scale,
+                                      const void* q, cascade_strides_t q_strides, const void* k,
+                                      cascade_strides_t k_strides, const void* v, cascade_strides_t v_strides,
+                                      void* o_out, cascade_strides_t o_strides, float* lse_out, void* workspace,
+                                      size_t workspace_bytes, void* stream) {
+  cascade_status_t s = check_attn_args("cascade_attn_sharded", plan, dtype, batch, n_heads, n_kv_heads,
+                                       head_dim, q, q_strides, k, k_strides, v, v_strides);
+  if (s != CASCADE_OK) return s;
+  if (!o_out) {
+    set_error("cascade_attn_sharded: null output pointer");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (!aligned16(o_out) || !strides_ok(o_strides, elt_size(dtype))) {
+    set_error("cascade_attn_sharded: output pointer and row strides must be 16-byte aligned");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  AttnParams p = make_params(plan, batch, n_heads, n_kv_heads, head_dim, scale, q, q_strides, k, k_strides, v,
+                             v_strides);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (use_decode(plan, dtype, n_heads, n_kv_heads, head_dim)) {
+    // one query row per sequence: every KV shard is an independent partial, combined by the merge kernel
+    const size_t need = decode_ws_bytes(plan, dtype, batch, n_heads, head_dim);
+    if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255)) {
+      set_error("cascade_attn_sharded: workspace of %zu bytes (256-byte aligned) required, got %zu", need,
+                workspace_bytes);
+      return CASCADE_ERR_WORKSPACE;
+    }
+    const size_t rows = (size_t)batch * plan->dev.n_kv_shards * plan->dev.n_q * n_heads;
+    char* ws = (char*)workspace;
+    p.fused = 0;
+    p.o_part = ws;
+    p.m_part = (float*)(ws + align_up(rows * head_dim * elt_size(dtype), 256));
+    p.l_part = (float*)((char*)p.m_part + align_up(rows * 4, 256));
+    cudaError_t e = launch_decode(p, st);
+    if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_sharded: decode launch");
+    MergeParams mp;
+    mp.o_part = p.o_part;
+    mp.m_part = p.m_part;
+    mp.l_part = p.l_part;
+    mp.row_scatter = nullptr;  // a single query row: slot 0 is token 0
+    mp.row_scatter_batch_stride = 0;
+    mp.o_out = o_out;
+    mp.os = {o_strides.batch, o_strides.token, o_strides.head};
+    mp.lse_out = lse_out;
+    mp.batch = batch;
+    mp.n_parts = plan->dev.n_kv_shards;
+    mp.n_rows = plan->dev.n_q;
+    mp.H = n_heads;
+    mp.d = head_dim;
+    e = launch_merge(mp, dtype, st);
+    if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_sharded: merge launch");
+    return CASCADE_OK;
+  }
+  p.fused = 1;
+  p.o_out = o_out;
+  p.os = {o_strides.batch, o_strides.token, o_strides.head};
+  p.lse_out = lse_out;
+  cudaError_t e = use_tc(plan, dtype, head_dim) ? launch_attn_tc(p, st) : launch_attn_simt(p, dtype, st);
+  if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_sharded: launch");
+  return CASCADE_OK;
+}
+
+}  // extern "C"

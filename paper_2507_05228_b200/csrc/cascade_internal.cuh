@@ -1,0 +1,90 @@
+// Internal declarations shared by the translation units of the CUDA library (not part of the ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "cascade.h"
+
+namespace cascade {
+
+// Device-side view of a plan.  All arrays have a leading n_maps dimension.
+struct PlanDev {
+  const int32_t* q_off;
+  const int32_t* q_idx;
+  const int32_t* q_inv;
+  const int32_t* kv_off;
+  const int32_t* kv_idx;
+  const int32_t* kv_inv;
+  const int32_t* vis;
+  const uint8_t* pair_class;
+  // Query tiles that never cross a shard boundary: {first slot, rows, shard, unused}; rows == 0 pads.
+  // Ordered by decreasing work (longest visible prefix first) so late CTAs are the short ones.
+  const int4* qtiles32;
+  const int4* qtiles128;
+  int32_t n_qtiles32;   // per map (padded to the maximum over maps)
+  int32_t n_qtiles128;
+  int32_t* status;      // device status word, 0 = fine
+  int32_t n_maps, n_q, n_kv, n_q_shards, n_kv_shards, q_pos_offset, causal;
+  int32_t max_kv_shard_len;
+};
+
+struct Strides {
+  int64_t batch, token, head;
+};
+
+struct AttnParams {
+  PlanDev plan;
+  const void* q;
+  const void* k;
+  const void* v;
+  Strides qs, ks, vs;
+  int32_t batch, H, Hkv, G, d;
+  float scale;
+  int32_t fused;  // 0: one job per KV shard, write (u, m, l); 1: walk all KV shards, write o (+lse)
+  void* o_part;
+  float* m_part;
+  float* l_part;
+  void* o_out;
+  Strides os;
+  float* lse_out;
+};
+
+struct MergeParams {
+  const void* o_part;
+  const float* m_part;
+  const float* l_part;
+  const int32_t* row_scatter;
+  int64_t row_scatter_batch_stride;
+  void* o_out;
+  Strides os;
+  float* lse_out;
+  int32_t batch, n_parts, n_rows, H, d;
+};
+
+}  // namespace cascade
+
+struct cascade_plan {
+  cascade::PlanDev dev;
+  std::vector<int32_t> q_off, q_idx, q_inv, kv_off, kv_idx, kv_inv, vis;
+  std::vector<uint8_t> pair_class;
+  std::vector<int4> qtiles32, qtiles128;
+  void* dev_blob = nullptr;
+  size_t dev_blob_bytes = 0;
+};
+
+namespace cascade {
+
+void set_error(const char* fmt, ...);
+void count_launch(int n = 1);
+
+// Launchers; each returns a cudaError_t from the launch.
+cudaError_t launch_attn_simt(const AttnParams& p, cascade_dtype_t dtype, cudaStream_t stream);
+cudaError_t launch_attn_tc(const AttnParams& p, cudaStream_t stream);
+cudaError_t launch_decode(const AttnParams& p, cudaStream_t stream);
+cudaError_t launch_merge(const MergeParams& p, cascade_dtype_t dtype, cudaStream_t stream);
+
+}  // namespace cascade

@@ -1,0 +1,165 @@
+"""GPU parity: the CUDA library through its C ABI against the fp64 oracle, element by element.
+
+Tolerances (max-abs on unit-variance Gaussian inputs with 1/sqrt(d) scaling): 2e-2 for bf16, 1e-4 for fp32,
+on partial outputs, merged outputs and fused outputs; same absolute bound on m and on m + ln l, relative bound
+|dl| <= tol * max(1, l) on l.  Plan arrays are compared bit-exactly.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2507_05228_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gu():
+    import gpu_util
+    return gpu_util
+
+
+def test_c1_tiny_fp32_full(gu):
+    gu.full_parity(wl.config("c1_tiny_f32"))
+
+
+def test_c2_prefill_8b_full(gu):
+    gu.full_parity(wl.config("c2_prefill_8b"))
+
+
+def test_c3_batched_reduced_and_outliers(gu):
+    gu.full_parity(wl.config("c3_batched", B=2, n_q=1024, n_kv=1024))
+
+
+def test_c3_batched_full_size_sampled(gu):
+    gu.sampled_parity(wl.config("c3_batched"), per_shard=1)
+
+
+def test_c4_long_reduced(gu):
+    gu.full_parity(wl.config("c4_long_70b", n_q=2048, n_kv=2048, H=16, Hkv=2))
+
+
+def test_c4_long_full_size_sampled(gu):
+    gu.sampled_parity(wl.config("c4_long_70b"), per_shard=1)
+
+
+def test_c5_decode_full(gu):
+    gu.full_parity(wl.config("c5_decode"))
+
+
+@pytest.mark.parametrize("dtype,d", [("f32", 64), ("f32", 128), ("bf16", 64), ("bf16", 128)])
+@pytest.mark.parametrize("H,Hkv", [(4, 4), (8, 2), (8, 1)])
+def test_ragged_shards_all_dtypes(gu, dtype, d, H, Hkv):
+    """Shard sizes from 1 to ~130 rows, N not a multiple of any tile, asymmetric query/KV maps, rows that see
+    nothing of some shard, an empty shard."""
+    rng = np.random.Generator(np.random.PCG64(d + H))
+    n = 517
+    sizes = [1, 2, 31, 33, 127, 129, 130, 64]  # sums to 517; shard 8 stays empty
+    assert sum(sizes) == n
+    kv_of = np.repeat(np.arange(8), sizes).astype(np.int32)
+    rng.shuffle(kv_of)
+    q_of = rng.integers(0, 5, n).astype(np.int32)
+    w = wl.make_workload("ragged", 2, n, n, H, Hkv, d, dtype, "random", "random", 5, 9, seed=77)
+    w.q_shard_of, w.kv_shard_of = q_of, kv_of
+    gu.full_parity(w)
+
+
+def test_contiguous_shards_have_empty_and_full_pairs(gu):
+    w = wl.make_workload("contig", 1, 640, 640, 8, 2, 128, "bf16", "contiguous", "contiguous", 5, 5, seed=5)
+    p = oracle.shard_plan(w.q_shard_of, w.kv_shard_of, 5, 5)
+    assert (p.pair_class == oracle.EMPTY).any() and (p.pair_class == oracle.FULL).any()
+    gu.full_parity(w)
+
+
+def test_non_causal_and_single_shard(gu):
+    gu.full_parity(wl.make_workload("bert_like", 2, 128, 128, 12, 12, 64, "f32", "round_robin", "round_robin",
+                                    4, 4, seed=3, causal=False))
+    gu.full_parity(wl.make_workload("one_shard", 1, 300, 300, 4, 2, 128, "bf16", "random", "random", 1, 1, seed=4))
+
+
+def test_chunked_prefill_offsets(gu):
+    """n_q < n_kv with the query block at the end of the cache, and a block in the middle."""
+    gu.full_parity(wl.make_workload("chunk_end", 2, 96, 400, 8, 2, 128, "bf16", "random", "random", 3, 7, seed=8))
+    gu.full_parity(wl.make_workload("chunk_mid", 1, 50, 333, 4, 4, 64, "f32", "round_robin", "random", 2, 5,
+                                    seed=9, q_pos_offset=100))
+
+
+@pytest.mark.parametrize("H,Hkv", [(8, 8), (8, 4), (32, 8), (16, 2)])
+def test_decode_group_sizes_and_ragged_cache(gu, H, Hkv):
+    w = wl.make_workload("decode_small", 3, 1, 1000, H, Hkv, 128, "bf16", "round_robin", "random", 1, 7, seed=H)
+    gu.full_parity(w)
+    # cache not fully visible (query position in the middle) and a shard with nothing visible
+    w2 = wl.make_workload("decode_partial", 2, 1, 500, H, Hkv, 128, "bf16", "round_robin", "contiguous", 1, 5,
+                          seed=H + 1, q_pos_offset=250)
+    gu.full_parity(w2)
+
+
+def test_per_sequence_maps_and_strided_inputs(gu):
+    from paper_2507_05228_b200 import binding as cb
+    B, n, H, Hkv, d = 3, 200, 8, 2, 128
+    w = wl.make_workload("perseq", B, n, n, H, Hkv, d, "bf16", "random", "random", 4, 4, seed=21)
+    rng = np.random.Generator(np.random.PCG64(5))
+    maps = np.stack([wl.shard_map("random", n, 4, rng) for _ in range(B)])
+    q, k, v = gu.to_device(w)
+    # pack q, k, v into one [B, n, H + 2 Hkv, d] tensor: strided views, as a fused QKV projection would give
+    packed = torch.cat([q, k, v], dim=2).contiguous()
+    qv, kv, vv = packed[:, :, :H], packed[:, :, H:H + Hkv], packed[:, :, H + Hkv:]
+    plan = cb.cascade_shard_plan(maps, maps, 4, 4)
+    o_part, m_part, l_part = cb.cascade_attn_partials(plan, qv, kv, vv, w.scale)
+    o_m, _ = cb.cascade_merge(o_part, m_part, l_part, plan.dev_ptr("q_idx"), row_scatter_batch_stride=n)
+    o_f, lse_f = cb.cascade_attn_sharded(plan, qv, kv, vv, w.scale)
+    o_ref, lse_ref = oracle.attention_unsharded(w.q, w.k, w.v, w.scale)
+    gu.check_output(o_m, None, o_ref, lse_ref, w.tol, "per-sequence maps merge")
+    gu.check_output(o_f, lse_f, o_ref, lse_ref, w.tol, "per-sequence maps fused")
+    for b in range(B):
+        op = oracle.shard_plan(maps[b], maps[b], 4, 4)
+        u, m, e = oracle.attn_pass(w.q[b:b + 1], w.k[b:b + 1], w.v[b:b + 1], w.scale, op)
+        gu.check_partials((o_part[b:b + 1].double().cpu().numpy(), m_part[b:b + 1].double().cpu().numpy(),
+                           l_part[b:b + 1].double().cpu().numpy()), (u, m, e), w.tol, f"per-sequence maps b={b}")
+    assert plan.device_status() == 0
+    plan.destroy()
+
+
+def test_merge_alone_matches_oracle_post_pass(gu):
+    """cascade_merge on synthetic partials (no attention involved), including empty parts and huge maxima."""
+    from paper_2507_05228_b200 import binding as cb
+    rng = np.random.Generator(np.random.PCG64(31))
+    for dtype, d, tol in ((torch.float32, 64, 1e-4), (torch.bfloat16, 128, 2e-2), (torch.float32, 128, 1e-4),
+                          (torch.bfloat16, 64, 2e-2)):
+        B, P, R, H = 2, 7, 37, 5
+        u = rng.standard_normal((B, P, R, H, d)).astype(np.float32)
+        if dtype == torch.bfloat16:
+            u = wl.round_to_bf16(u)
+        m = (rng.standard_normal((B, P, R, H)) * 30).astype(np.float32)
+        l = rng.uniform(1, 40, (B, P, R, H)).astype(np.float32)
+        dead = rng.random((B, P, R, H)) < 0.2
+        dead[0, :, 3, 1] = True  # a row whose parts are all empty
+        m[dead], l[dead] = -np.inf, 0.0
+        u[dead] = 0.0
+        scatter = rng.permutation(R).astype(np.int32)
+        o_ref, lse_ref = oracle.post_pass(u.astype(np.float64), m.astype(np.float64), l.astype(np.float64),
+                                          row_scatter=scatter)
+        sc = torch.from_numpy(scatter).cuda()
+        o, lse = cb.cascade_merge(torch.from_numpy(u).cuda().to(dtype), torch.from_numpy(m).cuda(),
+                                  torch.from_numpy(l).cuda(), sc.data_ptr())
+        gu.check_output(o, lse, o_ref, lse_ref, tol, f"merge {dtype} d={d}")
+        assert (o[0, scatter[3], 1] == 0).all() and torch.isneginf(lse[0, scatter[3], 1])
+
+
+def test_workspace_contract_for_decode(gu):
+    from paper_2507_05228_b200 import binding as cb
+    w = wl.make_workload("decode_ws", 2, 1, 256, 8, 2, 128, "bf16", "round_robin", "random", 1, 4, seed=2)
+    q, k, v = gu.to_device(w)
+    plan = gu.make_plan(w)
+    need = cb.cascade_workspace_bytes(plan, cb.CALL_SHARDED, cb.BF16, 2, 8, 2, 128)
+    assert need >= 2 * 4 * 8 * (128 * 2 + 8)
+    small = torch.empty(need - 256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(cb.CascadeError) as ei:
+        cb.cascade_attn_sharded(plan, q, k, v, w.scale, workspace=small)
+    assert ei.value.status == 4
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    o, _ = cb.cascade_attn_sharded(plan, q, k, v, w.scale, workspace=ws)
+    o_ref, lse_ref = oracle.attention_unsharded(w.q, w.k, w.v, w.scale, q_pos_offset=w.q_pos_offset)
+    gu.check_output(o, None, o_ref, lse_ref, w.tol, "decode with caller workspace")
+    plan.destroy()

@@ -1,0 +1,89 @@
+"""cascade_shard_plan's arrays against the oracle's, bit for bit (host-only plan: no GPU needed).
+The library builds them with a counting sort and binary searches; the oracle scans the mask definition."""
+import numpy as np
+import pytest
+
+import oracle
+from oracle import sharding
+from paper_2507_05228_b200 import workloads as wl
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2507_05228_b200 import build
+    build.build_library()
+    from paper_2507_05228_b200 import binding as b
+    return b
+
+
+def _compare(binding, q_of, kv_of, nq_s, nkv_s, off, causal):
+    ref = oracle.shard_plan(q_of, kv_of, nq_s, nkv_s, q_pos_offset=off, causal=causal)
+    plan = binding.cascade_shard_plan_host(q_of, kv_of, nq_s, nkv_s, q_pos_offset=off, causal=causal)
+    for f in ("q_off", "q_idx", "q_inv", "kv_off", "kv_idx", "kv_inv", "vis", "pair_class"):
+        got = plan.get(f)[0]
+        want = getattr(ref, f)
+        assert got.dtype == want.dtype and np.array_equal(got, want), f
+    return ref, plan
+
+
+@pytest.mark.parametrize("name", ["c1_tiny_f32", "c2_prefill_8b", "c3_batched", "c5_decode"])
+def test_plan_of_benchmark_maps_full_size(binding, name):
+    # only the maps matter here: shrink heads/batch so that no large tensor is drawn
+    w = wl.config(name, H=1, Hkv=1, B=1, d=8) if name != "c3_batched" else wl.config(name, H=1, Hkv=1, B=1, d=8,
+                                                                                        outlier_frac=0.0)
+    ref, plan = _compare(binding, w.q_shard_of, w.kv_shard_of, w.n_q_shards, w.n_kv_shards, w.q_pos_offset, True)
+    assert int(ref.vis.sum()) * 1 == w.visible_pairs()
+    j, k = w.n_q_shards - 1, 0
+    assert np.array_equal(plan.dense_mask(j, k), oracle.dense_mask(ref, j, k))
+    plan.destroy()
+
+
+def test_plan_of_long_context_map_full_size(binding):
+    w = wl.config("c4_long_70b", H=1, Hkv=1, d=8)
+    ref, plan = _compare(binding, w.q_shard_of, w.kv_shard_of, 32, 32, 0, True)
+    assert int(ref.vis.sum()) == 536887296
+    plan.destroy()
+
+
+def test_plan_random_maps_edge_cases(binding):
+    rng = np.random.Generator(np.random.PCG64(12))
+    for trial in range(60):
+        n_q, n_kv = int(rng.integers(1, 300)), int(rng.integers(1, 300))
+        nq_s, nkv_s = int(rng.integers(1, 9)), int(rng.integers(1, 12))
+        q_of = rng.integers(0, nq_s, n_q).astype(np.int32)
+        kv_of = rng.integers(0, nkv_s, n_kv).astype(np.int32)
+        if trial % 5 == 0:  # leave some shards empty, make one a single token
+            q_of[:] = 0
+            kv_of[:] = nkv_s - 1
+            kv_of[0] = 0
+        off = int(rng.integers(-5, n_kv + 5))
+        ref, plan = _compare(binding, q_of, kv_of, nq_s, nkv_s, off, causal=bool(trial % 4))
+        for j in range(nq_s):
+            for k in range(nkv_s):
+                assert np.array_equal(plan.dense_mask(j, k), oracle.dense_mask(ref, j, k))
+        plan.destroy()
+
+
+def test_plan_per_sequence_maps_and_paper_example(binding):
+    r_of = sharding.cdelta_shard_of(18, 2, 6)
+    s_of = sharding.m_split_shard_of(r_of, 2)
+    maps = np.stack([s_of, s_of[::-1].copy(), (np.arange(18) % 6).astype(np.int32)])
+    plan = binding.cascade_shard_plan_host(maps, maps, 6, 6)
+    for i in range(3):
+        ref = oracle.shard_plan(maps[i], maps[i], 6, 6)
+        assert np.array_equal(plan.get("q_idx")[i], ref.q_idx)
+        assert np.array_equal(plan.get("vis")[i], ref.vis)
+        assert np.array_equal(plan.get("pair_class")[i], ref.pair_class)
+    # Section 6.4 example: shard 0 = R_{1,1} = {1,7,13} (1-based)
+    assert (plan.get("q_idx")[0][:3] + 1).tolist() == [1, 7, 13]
+    plan.destroy()
+
+
+def test_partial_buffer_sizes_match_stage_b_cost_model():
+    """Appendix D: the partial outputs and statistics sent back are beta * (d + 2) * H * N values."""
+    w = wl.config("c2_prefill_8b", B=1, H=1, Hkv=1, d=8)
+    beta, d, H, N = 8, 128, 32, 2048
+    o_elems = beta * N * H * d
+    stat_elems = 2 * beta * N * H
+    assert o_elems + stat_elems == beta * (d + 2) * H * N
+    assert w.n_kv_shards == beta and w.n_q == N
