@@ -424,7 +424,7 @@ static bool use_decode(const cascade_plan_t* plan, cascade_dtype_t dtype, int H,
   return plan->dev.n_q == 1 && dtype == CASCADE_BF16 && d == 128 && (G == 1 || G == 2 || G == 4 || G == 8);
 }
 static bool use_tc(const cascade_plan_t* plan, cascade_dtype_t dtype, int d) {
-  return false && dtype == CASCADE_BF16 && d == 128 && plan->dev.n_q > 1;
+  return dtype == CASCADE_BF16 && d == 128 && plan->dev.n_q > 1;
 }
 
 static size_t decode_ws_bytes(const cascade_plan_t* plan, cascade_dtype_t dtype, int batch, int H, int d) {
