@@ -78,7 +78,7 @@ __device__ __noinline__ bool wait_slow(const WaitCtx& c, uint32_t bar, uint32_t 
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 255u) == 0) {
-      if (*c.abort_flag) return false;
+      if (*c.abort_flag || *reinterpret_cast<volatile int32_t*>(c.status) != 0) return false;
       if (global_timer_ns() - t0 > 2000000000ull) {
         *c.abort_flag = 1;
         atomicCAS(c.status, 0, code);
@@ -212,6 +212,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(AttnParams p) {
   const int4 qt = pl.qtiles128[(size_t)map * pl.n_qtiles128 + blockIdx.x];
   const int row0 = qt.x, nrows = qt.y;
   if (nrows == 0) return;  // padding entry (uniform for the CTA)
+  if (*reinterpret_cast<volatile int32_t*>(pl.status) != 0) return;  // an earlier CTA gave up: do not pile on
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int32_t* q_idx = pl.q_idx + (size_t)map * pl.n_q;
   const int32_t* kv_idx = pl.kv_idx + (size_t)map * pl.n_kv;
@@ -259,8 +260,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(AttnParams p) {
     float l_run = 0.f;
     int i = 0;  // flattened KV tile counter
     const bool row_ok = r < nrows;
-    uint32_t* sP = reinterpret_cast<uint32_t*>(smem + kOffP);
-    (void)sP;
     for (int kk = k_begin; kk < k_end; ++kk) {
       const int need = __ldg(vis_last + kk);
       const int full_upto = __ldg(vis_first + kk);
