@@ -180,6 +180,34 @@ cascade_status_t cascade_attn_sharded(const cascade_plan_t* plan, cascade_dtype_
                                       cascade_strides_t o_strides, float* lse_out, void* workspace,
                                       size_t workspace_bytes, void* stream);
 
+/*
+ * cascade_attn_decode_static -- the decode case of cascade_attn_sharded (one query row per sequence, bf16,
+ * head_dim 128, n_heads / n_kv_heads in {1,2,4,8}) without a workspace argument and without any allocation.
+ * (The paper has no counterpart: this is a convenience of this library, not a step of the method.)
+ *
+ * Who it is for: callers that cannot hand over scratch memory and cannot allocate it either -- a server whose
+ * cache manager already owns all free HBM, a decode loop that must not hit the device-wide synchronisation of
+ * cudaMalloc / cudaFree, a plug-in that only receives raw pointers.  The per-shard partials that the merge
+ * kernel combines live in a 16 MiB array compiled into the library (every GPU that loads the library carries
+ * it until the process exits).  The call issues no cudaMalloc, cudaFree or other allocating routine.
+ *
+ *  - Limit: batch * n_kv_shards * n_heads * 264 bytes (rounded up per region to 256) must fit in 16 MiB,
+ *    e.g. batch 64 x 16 shards x 32 heads = 8.3 MiB.  Larger problems return CASCADE_ERR_WORKSPACE with a
+ *    message naming the sizes; use cascade_attn_sharded with a workspace for those.
+ *  - The first call on each device looks up the array's device address (the device current at that moment).
+ *    Make that first call during start-up, before any stream capture.
+ *  - All calls share the one array.  Its contents are overwritten completely by each call before they are read,
+ *    so results never depend on an earlier call; but two calls whose kernels overlap on the GPU (different
+ *    streams, no ordering between them) race on it.  Keep calls on one stream or order them with events.
+ *  - Inputs, outputs, strides, stream and results are exactly those of cascade_attn_sharded.
+ */
+cascade_status_t cascade_attn_decode_static(const cascade_plan_t* plan, int32_t batch, int32_t n_heads,
+                                            int32_t n_kv_heads, float scale, const void* q,
+                                            cascade_strides_t q_strides, const void* k,
+                                            cascade_strides_t k_strides, const void* v,
+                                            cascade_strides_t v_strides, void* o_out, cascade_strides_t o_strides,
+                                            float* lse_out, void* stream);
+
 enum { CASCADE_CALL_PARTIALS = 0, CASCADE_CALL_SHARDED = 1 };
 
 /* Scratch bytes the given call needs for this plan and shape (0 if none).  The workspace must be

@@ -27,7 +27,7 @@ EXPORTS = [
     "cascade_version", "cascade_last_error", "cascade_launch_count", "cascade_shard_plan", "cascade_shard_plan_host",
     "cascade_plan_destroy",
     "cascade_plan_get", "cascade_plan_dense_mask", "cascade_plan_device_status", "cascade_attn_partials",
-    "cascade_merge", "cascade_attn_sharded", "cascade_workspace_bytes",
+    "cascade_merge", "cascade_attn_sharded", "cascade_workspace_bytes", "cascade_attn_decode_static",
 ]
 
 
@@ -68,6 +68,8 @@ def lib() -> ctypes.CDLL:
         L.cascade_merge.argtypes = [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, i64, vp, Strides, vp, vp]
         L.cascade_attn_sharded.argtypes = [vp, i32, i32, i32, i32, i32, f32, vp, Strides, vp, Strides, vp, Strides,
                                            vp, Strides, vp, vp, ctypes.c_size_t, vp]
+        L.cascade_attn_decode_static.argtypes = [vp, i32, i32, i32, f32, vp, Strides, vp, Strides, vp, Strides, vp,
+                                                 Strides, vp, vp]
         L.cascade_workspace_bytes.argtypes = [vp, i32, i32, i32, i32, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
         for name in EXPORTS:
             if name not in ("cascade_version", "cascade_last_error", "cascade_launch_count"):
@@ -259,4 +261,19 @@ def cascade_attn_sharded(plan: Plan, q: torch.Tensor, k: torch.Tensor, v: torch.
                                       k.data_ptr(), _strides(k), v.data_ptr(), _strides(v), o.data_ptr(),
                                       _strides(o), lse.data_ptr() if lse is not None else None, ws_ptr, ws_bytes,
                                       _stream()))
+    return o, lse
+
+
+def cascade_attn_decode_static(plan: Plan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, scale: float, out=None,
+                               want_lse: bool = True):
+    """Decode step (one query row per sequence) that uses the library's built-in 16 MiB scratch array instead of
+    a workspace: for callers that can neither pass nor allocate scratch memory.  Only the output tensors are
+    created here; the C call itself allocates nothing.  Returns (o [B, 1, H, 128], lse or None)."""
+    B, n_q, H, d = q.shape
+    assert n_q == 1 and d == 128 and q.dtype == torch.bfloat16
+    o = out if out is not None else torch.empty((B, n_q, H, d), dtype=q.dtype, device=q.device)
+    lse = torch.empty((B, n_q, H), dtype=torch.float32, device=q.device) if want_lse else None
+    _check(lib().cascade_attn_decode_static(plan.handle, B, H, k.shape[2], scale, q.data_ptr(), _strides(q),
+                                            k.data_ptr(), _strides(k), v.data_ptr(), _strides(v), o.data_ptr(),
+                                            _strides(o), lse.data_ptr() if lse is not None else None, _stream()))
     return o, lse
