@@ -10,9 +10,11 @@ struct Vec16;
 template <>
 struct Vec16<float> {
   static constexpr int N = 4;
-  static __device__ __forceinline__ void load(const float* p, float (&x)[4]) {
-    const float4 t = __ldcs(reinterpret_cast<const float4*>(p));
-    x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w;
+  using Raw = float4;
+  static __device__ __forceinline__ Raw load(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+  static __device__ __forceinline__ void fma(float (&acc)[4], const Raw& t, float w) {
+    acc[0] = fmaf(w, t.x, acc[0]); acc[1] = fmaf(w, t.y, acc[1]);
+    acc[2] = fmaf(w, t.z, acc[2]); acc[3] = fmaf(w, t.w, acc[3]);
   }
   static __device__ __forceinline__ void store(float* p, const float (&x)[4]) {
     *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
@@ -21,13 +23,14 @@ struct Vec16<float> {
 template <>
 struct Vec16<__nv_bfloat16> {
   static constexpr int N = 8;
-  static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&x)[8]) {
-    const uint4 t = __ldcs(reinterpret_cast<const uint4*>(p));
-    const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+  using Raw = uint4;
+  static __device__ __forceinline__ Raw load(const __nv_bfloat16* p) { return __ldcs(reinterpret_cast<const uint4*>(p)); }
+  static __device__ __forceinline__ void fma(float (&acc)[8], const Raw& t, float w) {
+    const uint32_t x[4] = {t.x, t.y, t.z, t.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      x[2 * i] = __uint_as_float(w[i] << 16);
-      x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+      acc[2 * i] = fmaf(w, __uint_as_float(x[i] << 16), acc[2 * i]);
+      acc[2 * i + 1] = fmaf(w, __uint_as_float(x[i] & 0xffff0000u), acc[2 * i + 1]);
     }
   }
   static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&x)[8]) {
@@ -41,66 +44,77 @@ struct Vec16<__nv_bfloat16> {
   }
 };
 
+// A group of TPR = D / (16 / sizeof(T)) lanes owns one (row, head) output vector.  The lanes share the work on the
+// statistics (lane `sub` evaluates the weights of parts sub, sub + TPR, ...; weights travel by shuffle) and each lane
+// streams its own 16 bytes of every partial with up to 8 loads in flight.
 template <typename T, int D>
-__global__ void __launch_bounds__(256) merge_kernel(MergeParams p) {
-  constexpr int V = Vec16<T>::N;
-  constexpr int TPR = D / V;       // threads per (row, head) vector
-  constexpr int ITEMS = 256 / TPR; // vectors per CTA
-  constexpr int CH = 4;            // parts fetched together
+__global__ void __launch_bounds__(256, 4) merge_kernel(MergeParams p) {
+  using VT = Vec16<T>;
+  constexpr int V = VT::N;
+  constexpr int TPR = D / V;
+  constexpr int ITEMS = 256 / TPR;
+  constexpr int CH = TPR < 8 ? TPR : 8;
   const int sub = threadIdx.x % TPR;
-  const int64_t item = (int64_t)blockIdx.x * ITEMS + threadIdx.x / TPR;
+  const int lane = threadIdx.x & 31;
+  const int group_lane0 = lane - sub;
   const int64_t per_batch = (int64_t)p.n_rows * p.H;
-  if (item >= per_batch * p.batch) return;
+  const int64_t total = per_batch * p.batch;
+  int64_t item = (int64_t)blockIdx.x * ITEMS + threadIdx.x / TPR;
+  const bool active = item < total;
+  if (!active) item = total - 1;  // keep the lane in the shuffles; it stores nothing
   const int b = (int)(item / per_batch);
   const int64_t rh = item - (int64_t)b * per_batch;  // r * H + h
   const int r = (int)(rh / p.H);
   const int h = (int)(rh - (int64_t)r * p.H);
-  const int64_t part_stride = per_batch;  // statistics per part
-  const float* mp = p.m_part + (int64_t)b * p.n_parts * part_stride + rh;
-  const float* lp = p.l_part + (int64_t)b * p.n_parts * part_stride + rh;
-  const T* up = static_cast<const T*>(p.o_part) + ((int64_t)b * p.n_parts * part_stride + rh) * D + sub * V;
+  const int P = p.n_parts;
+  const int64_t part_stride = per_batch;
+  const float* mp = p.m_part + (int64_t)b * P * part_stride + rh;
+  const float* lp = p.l_part + (int64_t)b * P * part_stride + rh;
+  const T* up = static_cast<const T*>(p.o_part) + ((int64_t)b * P * part_stride + rh) * D + sub * V;
 
   // line 3: n = max over parts of m
   float n = -INFINITY;
-  for (int k = 0; k < p.n_parts; ++k) n = fmaxf(n, __ldg(mp + (int64_t)k * part_stride));
+  for (int k = sub; k < P; k += TPR) n = fmaxf(n, __ldg(mp + (int64_t)k * part_stride));
+#pragma unroll
+  for (int off = TPR / 2; off > 0; off >>= 1) n = fmaxf(n, __shfl_xor_sync(0xffffffffu, n, off));
 
   float acc[V];
 #pragma unroll
   for (int i = 0; i < V; ++i) acc[i] = 0.f;
   float w = 0.f;
-  for (int k0 = 0; k0 < p.n_parts; k0 += CH) {
-    float u[CH][V];
-    float wt[CH];
-#pragma unroll
-    for (int c = 0; c < CH; ++c) {
-      const int k = k0 + c;
-      if (k < p.n_parts) {
-        Vec16<T>::load(up + (int64_t)k * part_stride * D, u[c]);
-        const float mk = __ldg(mp + (int64_t)k * part_stride);
-        const float lk = __ldg(lp + (int64_t)k * part_stride);
-        wt[c] = lk > 0.f ? expf(mk - n) * lk : 0.f;  // lines 5-6 weight; an empty part has l = 0
-      } else {
-        wt[c] = 0.f;
-#pragma unroll
-        for (int i = 0; i < V; ++i) u[c][i] = 0.f;
-      }
+  for (int base = 0; base < P; base += TPR) {
+    // lines 5-6: weight exp(m_k - n) * l_k of part base + sub (an empty part has l = 0)
+    float wt = 0.f;
+    if (base + sub < P) {
+      const float mk = __ldg(mp + (int64_t)(base + sub) * part_stride);
+      const float lk = __ldg(lp + (int64_t)(base + sub) * part_stride);
+      wt = lk > 0.f ? expf(mk - n) * lk : 0.f;
     }
+    w += wt;
+    const int cnt = min(TPR, P - base);  // warp-uniform
+    for (int c0 = 0; c0 < cnt; c0 += CH) {
+      typename VT::Raw u[CH];
 #pragma unroll
-    for (int c = 0; c < CH; ++c) {
-      w += wt[c];
-      if (wt[c] != 0.f) {
+      for (int c = 0; c < CH; ++c)
+        if (c0 + c < cnt) u[c] = VT::load(up + (int64_t)(base + c0 + c) * part_stride * D);
 #pragma unroll
-        for (int i = 0; i < V; ++i) acc[i] = fmaf(wt[c], u[c][i], acc[i]);
-      }
+      for (int c = 0; c < CH; ++c)
+        if (c0 + c < cnt) {
+          const float wc = __shfl_sync(0xffffffffu, wt, group_lane0 + c0 + c);
+          VT::fma(acc, u[c], wc);
+        }
     }
   }
+#pragma unroll
+  for (int off = TPR / 2; off > 0; off >>= 1) w += __shfl_xor_sync(0xffffffffu, w, off);
+  if (!active) return;
   const float inv = w > 0.f ? 1.f / w : 0.f;  // line 8
 #pragma unroll
   for (int i = 0; i < V; ++i) acc[i] *= inv;
   const int out_row = p.row_scatter ? __ldg(p.row_scatter + (int64_t)b * p.row_scatter_batch_stride + r) : r;
   T* op = static_cast<T*>(p.o_out) + (int64_t)b * p.os.batch + (int64_t)out_row * p.os.token +
           (int64_t)h * p.os.head + sub * V;
-  Vec16<T>::store(op, acc);
+  VT::store(op, acc);
   if (p.lse_out && sub == 0)
     p.lse_out[((int64_t)b * p.n_rows + out_row) * p.H + h] = w > 0.f ? n + logf(w) : -INFINITY;
 }
