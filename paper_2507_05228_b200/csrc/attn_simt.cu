@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(128) attn_simt_kernel(AttnParams p) {
   const int map = pl.n_maps == 1 ? 0 : b;
   const int h = blockIdx.y;
   const int g = h / p.G;
-  const int4 qt = pl.qtiles32[(size_t)map * pl.n_qtiles32 + blockIdx.x];
+  const int4 qt = pl.qtiles[0][(size_t)map * pl.n_qtiles[0] + blockIdx.x];
   const int row0 = qt.x, nrows = qt.y;
   if (nrows == 0) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -188,7 +188,7 @@ static cudaError_t launch_one(const AttnParams& p, dim3 grid, cudaStream_t strea
 
 cudaError_t launch_attn_simt(const AttnParams& p, cascade_dtype_t dtype, cudaStream_t stream) {
   const int n_parts = p.fused ? 1 : p.plan.n_kv_shards;
-  dim3 grid(p.plan.n_qtiles32, p.H, p.batch * n_parts);
+  dim3 grid(p.plan.n_qtiles[0], p.H, p.batch * n_parts);
   if (dtype == CASCADE_BF16) {
     if (p.d == 128) return launch_one<__nv_bfloat16, 128>(p, grid, stream);
     return launch_one<__nv_bfloat16, 64>(p, grid, stream);

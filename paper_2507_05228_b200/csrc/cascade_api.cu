@@ -165,22 +165,18 @@ static cascade_status_t plan_host(int32_t n_maps, int32_t n_q, int32_t n_kv, con
     }
     pl->dev.max_kv_shard_len = max_len;
     // tile lists, padded to the same length for every map
-    std::vector<std::vector<int4>> t32(n_maps), t128(n_maps);
-    size_t n32 = 0, n128 = 0;
-    for (int mp = 0; mp < n_maps; ++mp) {
-      build_qtiles(*pl, mp, 32, t32[mp]);
-      build_qtiles(*pl, mp, 128, t128[mp]);
-      n32 = std::max(n32, t32[mp].size());
-      n128 = std::max(n128, t128[mp].size());
+    for (int ts = 0; ts < kNumTileSizes; ++ts) {
+      std::vector<std::vector<int4>> lists(n_maps);
+      size_t n_max = 0;
+      for (int mp = 0; mp < n_maps; ++mp) {
+        build_qtiles(*pl, mp, 32 << ts, lists[mp]);
+        n_max = std::max(n_max, lists[mp].size());
+      }
+      pl->qtiles[ts].assign(n_max * n_maps, make_int4(0, 0, 0, 0));
+      for (int mp = 0; mp < n_maps; ++mp)
+        std::copy(lists[mp].begin(), lists[mp].end(), pl->qtiles[ts].begin() + mp * n_max);
+      pl->dev.n_qtiles[ts] = (int32_t)n_max;
     }
-    pl->qtiles32.assign(n32 * n_maps, make_int4(0, 0, 0, 0));
-    pl->qtiles128.assign(n128 * n_maps, make_int4(0, 0, 0, 0));
-    for (int mp = 0; mp < n_maps; ++mp) {
-      std::copy(t32[mp].begin(), t32[mp].end(), pl->qtiles32.begin() + mp * n32);
-      std::copy(t128[mp].begin(), t128[mp].end(), pl->qtiles128.begin() + mp * n128);
-    }
-    pl->dev.n_qtiles32 = (int32_t)n32;
-    pl->dev.n_qtiles128 = (int32_t)n128;
   } catch (const std::bad_alloc&) {
     delete pl;
     set_error("cascade_shard_plan: host allocation failed");
@@ -218,8 +214,10 @@ cascade_status_t cascade_shard_plan(int32_t n_maps, int32_t n_q, int32_t n_kv, c
       {pl->q_inv.data(), pl->q_inv.size() * 4, 0},       {pl->kv_off.data(), pl->kv_off.size() * 4, 0},
       {pl->kv_idx.data(), pl->kv_idx.size() * 4, 0},     {pl->kv_inv.data(), pl->kv_inv.size() * 4, 0},
       {pl->vis.data(), pl->vis.size() * 4, 0},           {pl->pair_class.data(), pl->pair_class.size(), 0},
-      {pl->qtiles32.data(), pl->qtiles32.size() * 16, 0}, {pl->qtiles128.data(), pl->qtiles128.size() * 16, 0},
+      {pl->qtiles[0].data(), pl->qtiles[0].size() * 16, 0}, {pl->qtiles[1].data(), pl->qtiles[1].size() * 16, 0},
+      {pl->qtiles[2].data(), pl->qtiles[2].size() * 16, 0}, {pl->qtiles[3].data(), pl->qtiles[3].size() * 16, 0},
   };
+  static_assert(kNumTileSizes == 4, "one upload segment per tile list");
   size_t total = 256;  // status word first
   for (auto& s : segs) {
     s.off = total;
@@ -252,8 +250,7 @@ cascade_status_t cascade_shard_plan(int32_t n_maps, int32_t n_q, int32_t n_kv, c
   pl->dev.kv_inv = (const int32_t*)(base + segs[5].off);
   pl->dev.vis = (const int32_t*)(base + segs[6].off);
   pl->dev.pair_class = (const uint8_t*)(base + segs[7].off);
-  pl->dev.qtiles32 = (const int4*)(base + segs[8].off);
-  pl->dev.qtiles128 = (const int4*)(base + segs[9].off);
+  for (int ts = 0; ts < kNumTileSizes; ++ts) pl->dev.qtiles[ts] = (const int4*)(base + segs[8 + ts].off);
   *out_plan = pl;
   return CASCADE_OK;
 }
@@ -331,11 +328,16 @@ cascade_status_t cascade_plan_device_status(const cascade_plan_t* plan, int32_t*
     set_error("cascade_plan_device_status: null pointer or host-only plan");
     return CASCADE_ERR_INVALID_ARG;
   }
+  int32_t words[20] = {0};
   cudaError_t e = cudaDeviceSynchronize();
-  if (e == cudaSuccess) e = cudaMemcpy(out_code, plan->dev.status, 4, cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess) e = cudaMemcpy(words, plan->dev.status, sizeof(words), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(e, "cascade_plan_device_status");
+  *out_code = words[0];
   if (*out_code != 0) {
-    set_error("device status word = %d: a bounded wait inside a kernel gave up", *out_code);
+    set_error("device status word = %d: a bounded wait inside a kernel gave up (block %d,%d,%d tile %d; warp progress "
+              "%d %d %d %d | %d %d %d %d | %d | %d %d %d)",
+              words[0], words[1], words[2], words[3], words[4], words[8], words[9], words[10], words[11], words[12],
+              words[13], words[14], words[15], words[16], words[17], words[18], words[19]);
     return CASCADE_ERR_TIMEOUT;
   }
   return CASCADE_OK;

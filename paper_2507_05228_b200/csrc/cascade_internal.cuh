@@ -11,6 +11,8 @@
 
 namespace cascade {
 
+constexpr int kNumTileSizes = 4;  // query-tile heights 32, 64, 128, 256
+
 // Device-side view of a plan.  All arrays have a leading n_maps dimension.
 struct PlanDev {
   const int32_t* q_off;
@@ -23,10 +25,9 @@ struct PlanDev {
   const uint8_t* pair_class;
   // Query tiles that never cross a shard boundary: {first slot, rows, shard, unused}; rows == 0 pads.
   // Ordered by decreasing work (longest visible prefix first) so late CTAs are the short ones.
-  const int4* qtiles32;
-  const int4* qtiles128;
-  int32_t n_qtiles32;   // per map (padded to the maximum over maps)
-  int32_t n_qtiles128;
+  // One list per tile height: qtiles[i] holds tiles of up to (32 << i) slots.
+  const int4* qtiles[kNumTileSizes];
+  int32_t n_qtiles[kNumTileSizes];  // per map (padded to the maximum over maps)
   int32_t* status;      // device status word, 0 = fine
   int32_t n_maps, n_q, n_kv, n_q_shards, n_kv_shards, q_pos_offset, causal;
   int32_t max_kv_shard_len;
@@ -71,7 +72,7 @@ struct cascade_plan {
   cascade::PlanDev dev;
   std::vector<int32_t> q_off, q_idx, q_inv, kv_off, kv_idx, kv_inv, vis;
   std::vector<uint8_t> pair_class;
-  std::vector<int4> qtiles32, qtiles128;
+  std::vector<int4> qtiles[cascade::kNumTileSizes];
   void* dev_blob = nullptr;
   size_t dev_blob_bytes = 0;
 };
