@@ -136,7 +136,9 @@ cascade_status_t cascade_plan_device_status(const cascade_plan_t* plan, int32_t*
  * per sequence, Appendix D.)  batch must equal n_maps when the plan has per-sequence maps.
  * head_dim in {64,128}; bf16 with head_dim 128 runs on the tensor cores (tcgen05), everything else on
  * the fp32 ALU kernel; n_q == 1 with bf16 runs the KV-streaming decode kernel.
- * workspace: as reported by cascade_workspace_bytes(CASCADE_CALL_PARTIALS) (may be 0 -> NULL allowed).
+ * workspace: as reported by cascade_workspace_bytes(CASCADE_CALL_PARTIALS) (may be 0 -> NULL allowed).  The
+ * tensor-core route first copies K and V into shard-major order there (the stage-A hand-over of each KV shard to
+ * its AttnNodes, Appendix D): 2 * batch * n_kv_heads * n_kv * head_dim * 2 bytes, overwritten by every call.
  */
 cascade_status_t cascade_attn_partials(const cascade_plan_t* plan, cascade_dtype_t dtype, int32_t batch,
                                        int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, float scale,
@@ -170,7 +172,8 @@ cascade_status_t cascade_merge(cascade_dtype_t dtype, int32_t batch, int32_t n_p
  * result equals cascade_merge(cascade_attn_partials(...)).  Output in token order:
  *   o_out [batch][n_q][n_heads][head_dim] with strides; lse_out optional fp32 [batch][n_q][n_heads].
  * For n_q == 1 (decode, Appendix F "Caching") the KV shards are processed as independent partials in
- * `workspace` and merged by a second launch.
+ * `workspace` and merged by a second launch.  The tensor-core route (bf16, head_dim 128) uses `workspace` for
+ * the shard-major K/V copies as cascade_attn_partials does.  Size: cascade_workspace_bytes(CASCADE_CALL_SHARDED).
  */
 cascade_status_t cascade_attn_sharded(const cascade_plan_t* plan, cascade_dtype_t dtype, int32_t batch,
                                       int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, float scale,

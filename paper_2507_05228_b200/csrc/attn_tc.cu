@@ -16,14 +16,23 @@
 //         tcgen05.ld, applies the shard mask (the row sees the first vis[slot][k] keys of the shard), keeps the running
 //         max / sum, writes the probabilities P as bf16 back into the TMEM columns of S, rescales the output
 //         accumulator in TMEM when the running max moved by more than 2^8, and runs the epilogue.
-//   8     MMA issuer (one lane): S_s = Q_s K^T (operands in shared memory) and O_s += P_s V (P from TMEM),
-//         issued as PV_0(i), QK_0(i+1), PV_1(i), QK_1(i+1) so that the tensor pipe works on one sub-tile while the
-//         other is in its softmax.  QK_s(i+1) overwrites the columns PV_s(i) reads P from; MMAs execute in issue
-//         order, which makes that safe without a barrier.
-//   9-11  loaders: index-mapped gather of 256-byte rows with 16-byte cp.async into the 128-byte-swizzled layout
-//         the MMA descriptors expect; warp 9 streams the K tiles, warps 10 and 11 the even and odd V tiles.
+//   8     MMA issuer: S_s = Q_s K^T (operands in shared memory) and O_s += P_s V (P from TMEM), issued as
+//         PV_0(i), QK_0(i+1), PV_1(i), QK_1(i+1) so that the tensor pipe works on one sub-tile while the other is in
+//         its softmax.  QK_s(i+1) overwrites the columns PV_s(i) reads P from; MMAs execute in issue order, which
+//         makes that safe without a barrier.  The whole warp runs the loop and one elected lane issues, so that
+//         descriptors and addresses stay warp-uniform.
+//   9-11  loaders, all TMA, completion counted in bytes on an mbarrier, data written in the 128-byte-swizzled layout
+//         the MMA descriptors expect.  Warp 9 streams the K tiles and warp 10 the V tiles from the shard-major
+//         copies that the gather pass (gather.cu) wrote: the visible prefix of a shard is a contiguous run of
+//         rows there, so a tile is two 16 KiB box loads.  Warp 11 brings the two query sub-tiles straight from
+//         the caller's tensor with index-mapped row gathers (tile::gather4: four rows of 128 bytes per
+//         instruction); that is done once per CTA only, a row gather being far too slow for the K/V stream
+//         (measured: one 512-byte gather per ~36 cycles per SM; 16-byte cp.async: one 512-byte request per ~90
+//         cycles per warp).
 // Every mbarrier wait is bounded: on expiry the CTA raises a flag, records a code in the plan's status word
 // and drains without waiting again.
+#include <cuda.h>
+
 #include "cascade_internal.cuh"
 
 namespace cascade {
@@ -41,6 +50,7 @@ constexpr uint32_t kTmemCols = 512;       // S0 | S1 | O0 | O1, 128 columns each
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 constexpr int kRegsSoftmax = 216;
 constexpr int kRegsOther = 72;
+constexpr int kMaxShardsInSmem = 96;      // per-shard prefix lengths are staged in shared memory up to this many
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int kOffQ = 0;
@@ -48,8 +58,9 @@ constexpr int kOffK = kOffQ + 2 * kTileBytes;
 constexpr int kOffV = kOffK + kKStages * kTileBytes;
 constexpr int kOffBar = kOffV + kVStages * kTileBytes;
 constexpr int kNumBars = 24;
-constexpr int kOffMisc = kOffBar + kNumBars * 8;
-constexpr int kSmemBytes = kOffMisc + 64 + 1024;  // + alignment slack
+constexpr int kOffMisc = kOffBar + kNumBars * 8;   // tmem slot, abort flag, 12 progress words
+constexpr int kOffShard = kOffMisc + 64;           // int32 [3][kMaxShardsInSmem]: need, first row of sub-tile 0 / 1
+constexpr int kSmemBytes = kOffShard + 3 * kMaxShardsInSmem * 4 + 1024;  // + alignment slack
 static_assert(kSmemBytes <= 232448, "exceeds the 227 KiB a CTA may use");
 
 enum Bar {
@@ -72,6 +83,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -87,6 +101,15 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
+}
+__device__ __forceinline__ bool elect_one() {  // true in exactly one lane of a converged warp
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
 }
 
 struct WaitCtx {
@@ -122,27 +145,35 @@ __device__ __forceinline__ bool wait_bar(const WaitCtx& c, uint32_t bar, uint32_
   return true;
 }
 
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+// TMA row gather: rows r0..r3 of the 2-D tensor, 64 elements (128 bytes) starting at column `col`, land as four
+// consecutive 128-byte rows at `dst` (swizzled by the hardware according to the shared-memory address).
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map, int col, int r0, int r1, int r2,
+                                            int r3, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cta.global.tile::gather4.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(col), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar)
+      : "memory");
 }
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+// TMA box load: 128 rows x 64 elements of the 3-D tensor [matrix z][row y][column x] land as 128 rows of 128 bytes.
+__device__ __forceinline__ void tma_tile3(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar)
+      : "memory");
 }
 
-// Shared-memory matrix descriptor, 128-byte swizzle.  Fields: start address >> 4 (bits 0-13), leading-dimension
-// byte offset >> 4 (16-29), stride-dimension byte offset >> 4 (32-45), descriptor version 1 (46-47), layout
-// type 2 = SWIZZLE_128B (61-63).
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
-         ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+// Shared-memory matrix descriptor, 128-byte swizzle, as two 32-bit words.  Low word: start address >> 4 (bits 0-13),
+// leading-dimension byte offset >> 4 (bits 16-29).  High word: stride-dimension byte offset >> 4 (bits 0-13),
+// descriptor version 1 (bits 14-15), layout type 2 = SWIZZLE_128B (bits 29-31).  Stepping along K only changes the
+// start address, so the issuing code adds small constants to a precomputed low word.
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+  return ((saddr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
 }
+__host__ __device__ constexpr uint32_t desc_hi(uint32_t sbo_bytes) { return (sbo_bytes >> 4) | (1u << 14) | (2u << 29); }
 // Instruction descriptor for kind::f16: D fp32 (bits 4-5 = 1), A and B bf16 (bits 7-9, 10-12 = 1), operand
 // majors (bit 15 A, bit 16 B; 0 = K-major, 1 = MN-major), N >> 3 at bits 17-22, M >> 4 at bits 24-28.
 __host__ __device__ constexpr uint32_t make_idesc(int m, int n, int a_mn_major, int b_mn_major) {
@@ -150,24 +181,27 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n, int a_mn_major, 
          ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
+// D[tmem] (+)= A[smem] * B[smem]; both descriptors share the high word
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                       bool accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"((uint32_t)accumulate)
       : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]; A is 128 lanes x 8 columns, each column holding two consecutive bf16 along K
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                       bool accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"((uint32_t)accumulate)
       : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
@@ -222,27 +256,40 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
   return y;
 }
-
+// two fp32 lanes in one 64-bit register (packed FMA / ADD halve the issue slots of the exponent loop)
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-// Byte offset of 16-byte chunk `chunk` (0..15) of row `row` inside a [2][128][128 B] swizzled tile.
-__device__ __forceinline__ uint32_t tile_offset(int row, int chunk) {
-  return (uint32_t)((chunk >> 3) * kHalfBytes + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
-}
-
 // The CTA's sequence of KV tiles: shard by shard, each shard's visible prefix (as seen by the CTA's last row, which
 // has the longest one) in pieces of at most 128 keys.  Every role walks the same sequence.
 struct TileWalk {
-  const int32_t* need_of;  // vis[last row of the CTA][*]
+  const int32_t* need_of;  // vis[last row of the CTA][*] (shared-memory copy when it fits)
   int k_end, kk, t0, need;
   __device__ __forceinline__ void seek() {
     t0 = 0;
     need = 0;
     while (kk < k_end) {
-      need = __ldg(need_of + kk);
+      need = need_of[kk];
       if (need > 0) break;
       ++kk;
     }
@@ -265,24 +312,18 @@ struct TileWalk {
   }
 };
 
-// One warp gathers rows [0, n_rows) of a tile (n_rows a multiple of 32).  tok_of(row) returns the source token of the
-// row or -1 for a zero-filled row; src_of(row, tok) returns the address of the row's 256 bytes.
-template <typename TokOf, typename SrcOf>
-__device__ __forceinline__ void gather_rows(uint32_t tile_saddr, int n_rows, int lane, TokOf tok_of, SrcOf src_of) {
-  const int chunk = lane & 15, sub = lane >> 4;
-  for (int r0 = 0; r0 < n_rows; r0 += 32) {
-    const int my_tok = tok_of(r0 + lane);  // one coalesced index load per 32 rows
-#pragma unroll
-    for (int pp = 0; pp < 16; ++pp) {
-      const int row = r0 + 2 * pp + sub;
-      const int tok = __shfl_sync(0xffffffffu, my_tok, 2 * pp + sub);
-      const bool ok = tok >= 0;
-      cp_async16(tile_saddr + tile_offset(row, chunk), src_of(row, ok ? tok : 0) + chunk * 8, ok ? 16u : 0u);
-    }
-  }
-}
+// How a (batch, token, head) triple maps to a row of the 2-D view [rows][head_dim] a row-gather tensor map describes.
+struct RowMap {
+  int32_t per_batch, per_token, per_head;
+};
+struct TmaArgs {
+  CUtensorMap q;     // the caller's query tensor as [rows][head_dim]
+  CUtensorMap k, v;  // shard-major copies as [batch * kv_heads][n_kv][head_dim]
+  RowMap qr;
+};
 
-__global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(AttnParams p, int lg) {
+__global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_constant__ AttnParams p, int lg,
+                                                              const __grid_constant__ TmaArgs tma) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -291,6 +332,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(AttnParams p, int 
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kOffMisc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffMisc + 4);
   volatile int* progress = reinterpret_cast<volatile int*>(smem + kOffMisc + 8);  // [12]
+  int32_t* shard_tab = reinterpret_cast<int32_t*>(smem + kOffShard);              // [3][kMaxShardsInSmem]
 
   // lg = log2(Gp): Gp heads stacked per tile, R = 128 / Gp slots per sub-tile, 2 R slots per CTA
   const int Gp = 1 << lg, R = kM >> lg;
@@ -310,25 +352,37 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(AttnParams p, int 
   const int n_sub = nrows > R ? 2 : 1;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int32_t* q_idx = pl.q_idx + (size_t)map * pl.n_q;
-  const int32_t* kv_idx = pl.kv_idx + (size_t)map * pl.n_kv;
   const int32_t* kv_off = pl.kv_off + (size_t)map * (P + 1);
   const int32_t* vis = pl.vis + (size_t)map * pl.n_q * P;
-  const int32_t* vis_last = vis + (size_t)(row0 + nrows - 1) * P;  // longest prefix of the CTA (rows ascend)
   const int k_begin = p.fused ? 0 : part, k_end = p.fused ? P : part + 1;
+  // Per-shard prefix lengths the roles consult at every shard change: the CTA's last row (longest prefix, drives the
+  // tile walk) and the first row of each sub-tile (shortest prefix, decides whether a tile needs the mask).
+  const int32_t* need_of = vis + (size_t)(row0 + nrows - 1) * P;
+  const int32_t* first_of[2] = {vis + (size_t)row0 * P, vis + (size_t)(row0 + (n_sub - 1) * R) * P};
+  if (P <= kMaxShardsInSmem) {
+    for (int kk = tid; kk < P; kk += kThreads) {
+      shard_tab[kk] = __ldg(need_of + kk);
+      shard_tab[kMaxShardsInSmem + kk] = __ldg(first_of[0] + kk);
+      shard_tab[2 * kMaxShardsInSmem + kk] = __ldg(first_of[1] + kk);
+    }
+    need_of = shard_tab;
+    first_of[0] = shard_tab + kMaxShardsInSmem;
+    first_of[1] = shard_tab + 2 * kMaxShardsInSmem;
+  }
   WaitCtx wc{abort_flag, progress, pl.status};
   auto note = [&](int v) {
     if (lane == 0) progress[warp] = v;
   };
 
   if (tid == 0) {
-    mbar_init(bar(Q_FULL), 32);
-    mbar_init(bar(Q_FULL + 1), 32);
+    mbar_init(bar(Q_FULL), 1);  // the *_FULL barriers: one arrival that announces the byte count, then the bytes
+    mbar_init(bar(Q_FULL + 1), 1);
     for (int s = 0; s < kKStages; ++s) {
-      mbar_init(bar(K_FULL + s), 32);
+      mbar_init(bar(K_FULL + s), 1);
       mbar_init(bar(K_EMPTY + s), 1);
     }
     for (int s = 0; s < kVStages; ++s) {
-      mbar_init(bar(V_FULL + s), 32);
+      mbar_init(bar(V_FULL + s), 1);
       mbar_init(bar(V_EMPTY + s), 1);
     }
     for (int s = 0; s < 2; ++s) {
@@ -365,21 +419,29 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(AttnParams p, int 
       const int slot = sub_row0 + (row_ok ? slot_local : 0);
       const int head = h0 + (m & (Gp - 1));
       const int32_t* vis_row = vis + (size_t)slot * P;
-      const int32_t* vis_first = vis + (size_t)sub_row0 * P;  // shortest prefix of the sub-tile
+      const int32_t* vis_first = first_of[s];  // shortest prefix of the sub-tile
       const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
       const uint32_t s_addr = lane_base + (uint32_t)(s * 128);
       const uint32_t o_addr = lane_base + 256u + (uint32_t)(s * 128);
       const float c = p.scale * 1.4426950408889634f;  // logits are kept in log2 units: x = s * scale * log2(e)
+      const uint64_t c2 = pack2(c, c);
       float m_run = -INFINITY;   // reference max the accumulators are scaled by (may lag by < 2^8)
       float m_true = -INFINITY;  // exact running max
       float l_run = 0.f;
       int my_vis = 0, full_upto = 0;
       int i = 0;  // KV tile counter
       TileWalk w;
-      for (w.start(vis_last, k_begin, k_end); !w.done(); w.next(), ++i) {
+      w.start(need_of, k_begin, k_end);
+      // this row's prefix length in the shard being walked, fetched one shard ahead
+      int vis_next = (!w.done() && row_ok) ? __ldg(vis_row + w.kk) : 0;
+      for (; !w.done(); w.next(), ++i) {
         if (w.t0 == 0) {  // entered a new shard
-          my_vis = row_ok ? __ldg(vis_row + w.kk) : 0;
-          full_upto = __ldg(vis_first + w.kk);
+          my_vis = vis_next;
+          full_upto = vis_first[w.kk];
+          TileWalk peek = w;  // the next shard with something visible
+          ++peek.kk;
+          peek.seek();
+          vis_next = (!peek.done() && row_ok) ? __ldg(vis_row + peek.kk) : 0;
         }
         const int n = w.n();
         const int nch = n >> 5;
@@ -392,29 +454,30 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(AttnParams p, int 
         if (nch > 2) CASCADE_TMEM_LD32(s_addr + 64, sr, 64);
         if (nch > 3) CASCADE_TMEM_LD32(s_addr + 96, sr, 96);
         tmem_wait_ld();
-        // mask (only tiles that reach past the shortest prefix of the sub-tile need it) and tile max
-        float tmax;
-        if (n == kNMax && w.t0 + n <= full_upto) {  // every valid row of the sub-tile sees all 128 keys
-          float mx[4];
+        // mask: only tiles that reach past the shortest prefix of the sub-tile need it.  Columns [0, lim) are visible
+        // to this row (lim <= keys <= n, so this also covers columns that were never loaded).  The mask is applied
+        // through a per-chunk bit mask so that the compiler can move several bits at a time into predicates.
+        if (!(n == kNMax && w.t0 + n <= full_upto)) {
+          const int lim = my_vis - w.t0;
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            mx[q4] = __uint_as_float(sr[32 * q4]);
+          for (int ch = 0; ch < 4; ++ch) {
+            const int lc = lim - 32 * ch;
+            const uint32_t mk = lc >= 32 ? 0xffffffffu : (lc <= 0 ? 0u : ((1u << lc) - 1u));
 #pragma unroll
-            for (int j = 1; j < 31; j += 2)
-              mx[q4] = fmax3(mx[q4], __uint_as_float(sr[32 * q4 + j]), __uint_as_float(sr[32 * q4 + j + 1]));
-            mx[q4] = fmaxf(mx[q4], __uint_as_float(sr[32 * q4 + 31]));
-          }
-          tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-        } else {
-          const int lim = my_vis - w.t0;  // columns [0, lim) are visible to this row; lim <= keys <= n
-          tmax = -INFINITY;
-#pragma unroll
-          for (int j = 0; j < 128; ++j) {
-            if (j >= lim) sr[j] = 0xff800000u;  // -inf (also covers the columns that were never loaded)
-            tmax = fmaxf(tmax, __uint_as_float(sr[j]));
+            for (int j = 0; j < 32; ++j)
+              if (!((mk >> j) & 1u)) sr[32 * ch + j] = 0xff800000u;  // -inf
           }
         }
-        tmax *= c;
+        float mx[4];
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+          mx[q4] = __uint_as_float(sr[32 * q4]);
+#pragma unroll
+          for (int j = 1; j < 31; j += 2)
+            mx[q4] = fmax3(mx[q4], __uint_as_float(sr[32 * q4 + j]), __uint_as_float(sr[32 * q4 + j + 1]));
+          mx[q4] = fmaxf(mx[q4], __uint_as_float(sr[32 * q4 + 31]));
+        }
+        const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c;
         m_true = fmaxf(m_true, tmax);
         float m_new = m_run;
         if (m_run == -INFINITY || m_true > m_run + kRescaleThreshold) m_new = m_true;
@@ -422,23 +485,27 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(AttnParams p, int 
         const bool changed = m_new != m_run;
         m_run = m_new;
         const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
-        float psum0 = 0.f, psum1 = 0.f;
+        const uint64_t neg_m2 = pack2(neg_m, neg_m);
+        uint64_t psum2 = pack2(0.f, 0.f);
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
           if (ch < nch) {  // warp-uniform
             uint32_t pk[16];
 #pragma unroll
             for (int j = 0; j < 32; j += 2) {
-              const float p0 = ex2(fmaf(__uint_as_float(sr[32 * ch + j]), c, neg_m));
-              const float p1 = ex2(fmaf(__uint_as_float(sr[32 * ch + j + 1]), c, neg_m));
-              psum0 += p0;
-              psum1 += p1;
+              float x0, x1;
+              unpack2(ffma2(pack2(__uint_as_float(sr[32 * ch + j]), __uint_as_float(sr[32 * ch + j + 1])), c2, neg_m2),
+                      x0, x1);
+              const float p0 = ex2(x0), p1 = ex2(x1);
+              psum2 = fadd2(psum2, pack2(p0, p1));
               pk[j >> 1] = pack_bf16x2(p0, p1);
             }
             // P as the A operand of the PV product: lane = row, column kk holds keys 2 kk and 2 kk + 1
             CASCADE_TMEM_ST16(s_addr + (uint32_t)(16 * ch), pk);
           }
         }
+        float psum0, psum1;
+        unpack2(psum2, psum0, psum1);
         l_run = l_run * alpha + (psum0 + psum1);
         // S_FULL(i) was committed after PV(i-1), so the output accumulator is quiescent until this thread's
         // arrival on P_FULL(i) below
@@ -516,137 +583,139 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(AttnParams p, int 
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
     if (warp == 8) {
       // ---------------------------------------------------------------- MMA issuer
-      if (lane == 0) {
-        constexpr uint32_t idesc_pv = make_idesc(kM, kD, 0, 1);
-        const uint32_t q_s = smem_base + kOffQ;
-        TileWalk w;
-        w.start(vis_last, k_begin, k_end);
-        if (!w.done()) {
-          auto issue_qk = [&](int s, int i, int n) {  // S_s = Q_s K(i)^T, n keys wide
-            const uint32_t k_s = smem_base + kOffK + (i % kKStages) * kTileBytes;
-            const uint32_t idesc_qk = make_idesc(kM, n, 0, 0);
+      // All 32 lanes run the loop (waits included) so that every address and descriptor is warp-uniform; the
+      // tcgen05 instructions themselves are issued by one elected lane.
+      const bool leader = elect_one();
+      constexpr uint32_t idesc_pv = make_idesc(kM, kD, 0, 1);
+      constexpr uint32_t hi_kmajor = desc_hi(1024);  // Q, K: 8-row groups 1024 bytes apart
+      constexpr uint32_t hi_v = desc_hi(1024);       // V (MN-major): 8-key groups 1024 bytes apart
+      const uint32_t q_lo0 = desc_lo(smem_base + kOffQ, 16);
+      const uint32_t k_lo0 = desc_lo(smem_base + kOffK, 16);
+      const uint32_t v_lo0 = desc_lo(smem_base + kOffV, kHalfBytes);  // the two 64-column halves of d
+      TileWalk w;
+      w.start(need_of, k_begin, k_end);
+      if (!w.done()) {
+        auto issue_qk = [&](int s, int i, int n) {  // S_s = Q_s K(i)^T, n keys wide
+          const uint32_t q_lo = q_lo0 + (uint32_t)(s * (kTileBytes >> 4));
+          const uint32_t k_lo = k_lo0 + (uint32_t)((i % kKStages) * (kTileBytes >> 4));
+          const uint32_t idesc_qk = make_idesc(kM, n, 0, 0);
+          if (leader) {
 #pragma unroll
             for (int ks = 0; ks < kD / 16; ++ks) {
-              const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-              mma_ss(tmem + (uint32_t)(s * 128), make_desc(q_s + s * kTileBytes + off, 16, 1024),
-                     make_desc(k_s + off, 16, 1024), idesc_qk, ks > 0 ? 1u : 0u);
+              // 16 elements of head_dim = 32 bytes along the 128-byte row; elements 64.. live in the second half
+              const uint32_t off = (uint32_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
+              mma_ss(tmem + (uint32_t)(s * 128), q_lo + off, k_lo + off, hi_kmajor, idesc_qk, ks > 0);
             }
             mma_commit(bar(S_FULL + s));
-          };
-          auto issue_pv = [&](int s, int i, int n) {  // O_s (+)= P_s V(i) over n keys
-            const uint32_t v_s = smem_base + kOffV + (i % kVStages) * kTileBytes;
-            const int ksteps = n >> 4;
-            for (int ks = 0; ks < ksteps; ++ks) {
+          }
+        };
+        auto issue_pv = [&](int s, int i, int n) {  // O_s (+)= P_s V(i) over n keys
+          const uint32_t v_lo = v_lo0 + (uint32_t)((i % kVStages) * (kTileBytes >> 4));
+          const int ksteps = n >> 4;
+          if (leader) {
+#pragma unroll
+            for (int ks = 0; ks < kNMax / 16; ++ks) {
               // A = P from TMEM: 16 keys = 8 columns; B = V (MN-major): 16 keys = 16 rows of 128 bytes
-              mma_ts(tmem + 256u + (uint32_t)(s * 128), tmem + (uint32_t)(s * 128 + ks * 8),
-                     make_desc(v_s + ks * 2048, kHalfBytes, 1024), idesc_pv, (i > 0 || ks > 0) ? 1u : 0u);
+              if (ks < ksteps)
+                mma_ts(tmem + 256u + (uint32_t)(s * 128), tmem + (uint32_t)(s * 128 + ks * 8),
+                       v_lo + (uint32_t)(ks * (2048 >> 4)), hi_v, idesc_pv, i > 0 || ks > 0);
             }
-          };
-          int n_cur = w.n();
-          wait_bar(wc, bar(K_FULL), 0u, 7);
-          for (int s = 0; s < n_sub; ++s) {
-            wait_bar(wc, bar(Q_FULL + s), 0u, 6);
-            tc_fence_after();
-            issue_qk(s, 0, n_cur);
           }
-          mma_commit(bar(K_EMPTY));
-          w.next();
-          for (int i = 0;; ++i) {
-            const bool has_next = !w.done();
-            const int n_next = has_next ? w.n() : 0;
-            progress[warp] = 8 * i + 1;
-            wait_bar(wc, bar(V_FULL + i % kVStages), (uint32_t)((i / kVStages) & 1), 4, i);
-            for (int s = 0; s < n_sub; ++s) {
-              progress[warp] = 8 * i + 2 + s;
-              wait_bar(wc, bar(P_FULL + s), (uint32_t)(i & 1), 5, i);
-              tc_fence_after();
-              issue_pv(s, i, n_cur);
-              if (s == n_sub - 1) mma_commit(bar(V_EMPTY + i % kVStages));
-              if (has_next) {
-                if (s == 0) {
-                  progress[warp] = 8 * i + 4;
-                  wait_bar(wc, bar(K_FULL + (i + 1) % kKStages), (uint32_t)(((i + 1) / kKStages) & 1), 7, i);
-                  tc_fence_after();
-                }
-                issue_qk(s, i + 1, n_next);
-                if (s == n_sub - 1) mma_commit(bar(K_EMPTY + (i + 1) % kKStages));
-              }
-            }
-            if (!has_next) break;
-            n_cur = n_next;
-            w.next();
-          }
-          mma_commit(bar(O_FULL));
-          progress[warp] = 7;
+        };
+        int n_cur = w.n();
+        wait_bar(wc, bar(K_FULL), 0u, 7);
+        for (int s = 0; s < n_sub; ++s) {
+          wait_bar(wc, bar(Q_FULL + s), 0u, 6);
+          tc_fence_after();
+          issue_qk(s, 0, n_cur);
         }
+        if (leader) mma_commit(bar(K_EMPTY));
+        w.next();
+        for (int i = 0;; ++i) {
+          const bool has_next = !w.done();
+          const int n_next = has_next ? w.n() : 0;
+          note(8 * i + 1);
+          wait_bar(wc, bar(V_FULL + i % kVStages), (uint32_t)((i / kVStages) & 1), 4, i);
+          for (int s = 0; s < n_sub; ++s) {
+            note(8 * i + 2 + s);
+            wait_bar(wc, bar(P_FULL + s), (uint32_t)(i & 1), 5, i);
+            tc_fence_after();
+            issue_pv(s, i, n_cur);
+            if (s == n_sub - 1 && leader) mma_commit(bar(V_EMPTY + i % kVStages));
+            if (has_next) {
+              if (s == 0) {
+                note(8 * i + 4);
+                wait_bar(wc, bar(K_FULL + (i + 1) % kKStages), (uint32_t)(((i + 1) / kKStages) & 1), 7, i);
+                tc_fence_after();
+              }
+              issue_qk(s, i + 1, n_next);
+              if (s == n_sub - 1 && leader) mma_commit(bar(K_EMPTY + (i + 1) % kKStages));
+            }
+          }
+          if (!has_next) break;
+          n_cur = n_next;
+          w.next();
+        }
+        if (leader) mma_commit(bar(O_FULL));
+        note(7);
       }
       __syncwarp();
     } else {
       // ---------------------------------------------------------------- loaders
       // Every barrier is served by one warp only, in tile order: a phase-parity wait cannot tell "one phase behind"
       // from "one phase ahead", so a warp must never skip a use of a stage.
-      //   warp 9: all K tiles, two gathers in flight (K(i) is announced once K(i+1) has been issued)
-      //   warp 10: Q_0, then V(0), V(2), ...;  warp 11: Q_1, then V(1), V(3), ...   (V stage = tile parity)
+      //   warp 9: the K tiles, warp 10: the V tiles, warp 11: the query sub-tiles.
       const int lw = warp - 9;
-      const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(p.k) + (int64_t)b * p.ks.batch + (int64_t)g * p.ks.head;
-      const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(p.v) + (int64_t)b * p.vs.batch + (int64_t)g * p.vs.head;
-      const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(p.q) + (int64_t)b * p.qs.batch + (int64_t)h0 * p.qs.head;
       TileWalk w;
-      w.start(vis_last, k_begin, k_end);
+      w.start(need_of, k_begin, k_end);
       if (!w.done()) {
-        if (lw >= 1 && lw - 1 < n_sub) {  // query sub-tile (row m = slot m / Gp, head m % Gp)
-          const int s = lw - 1;
-          const int sub_row0 = row0 + s * R;
-          const int sub_nrows = min(R, nrows - s * R);
-          gather_rows(
-              smem_base + kOffQ + s * kTileBytes, kM, lane,
-              [&](int row) { return (row >> lg) < sub_nrows ? __ldg(q_idx + sub_row0 + (row >> lg)) : -1; },
-              [&](int row, int tok) { return qb + (int64_t)tok * p.qs.token + (int64_t)(row & (Gp - 1)) * p.qs.head; });
-          cp_async_wait_all();
-          fence_proxy_async();
-          mbar_arrive(bar(Q_FULL + s));
-        }
-        int i = 0;
-        int announced = -1;  // K stage whose gather has been issued but not yet announced
-        for (; !w.done(); w.next(), ++i) {
-          const int keys = w.keys(), n = w.n();
-          const int32_t* idx = kv_idx + __ldg(kv_off + w.kk) + w.t0;
-          auto tok_of = [&](int row) { return row < keys ? __ldg(idx + row) : -1; };
-          if (lw == 0) {
-            const int st = i % kKStages;
-            note(8 * i + 1);
-            wait_bar(wc, bar(K_EMPTY + st), (uint32_t)(((i / kKStages) & 1) ^ 1), 9, i);
-            gather_rows(smem_base + kOffK + st * kTileBytes, n, lane, tok_of,
-                        [&](int, int tok) { return kb + (int64_t)tok * p.ks.token; });
-            cp_async_commit();
-            if (announced >= 0) {
-              cp_async_wait<1>();  // everything but the gather just issued has landed
-              fence_proxy_async();
-              mbar_arrive(bar(K_FULL + announced));
+        if (lw == 2) {
+          // Query rows: row m of the sub-tile = slot m / Gp, head m % Gp; lane l brings rows 4 l .. 4 l + 3, the two
+          // 128-byte halves of head_dim with one gather each.  Rows past the end of a sub-tile repeat its last
+          // row (their results are discarded), so no out-of-range coordinate is ever used.
+          for (int s = 0; s < n_sub; ++s) {
+            const int sub_row0 = row0 + s * R;
+            const int sub_nrows = min(R, nrows - s * R);
+            int r[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int m = 4 * lane + j;
+              const int tok = __ldg(q_idx + sub_row0 + min(m >> lg, sub_nrows - 1));
+              r[j] = b * tma.qr.per_batch + tok * tma.qr.per_token + (h0 + (m & (Gp - 1))) * tma.qr.per_head;
             }
-            announced = st;
+            const uint32_t fb = bar(Q_FULL + s);
+            if (lane == 0) mbar_expect_tx(fb, (uint32_t)kTileBytes);
+            __syncwarp();
+            const uint32_t dst = smem_base + kOffQ + (uint32_t)(s * kTileBytes + 4 * lane * 128);
+            tma_gather4(dst, &tma.q, 0, r[0], r[1], r[2], r[3], fb);
+            tma_gather4(dst + kHalfBytes, &tma.q, 64, r[0], r[1], r[2], r[3], fb);
+          }
+        } else {
+          const bool is_k = lw == 0;
+          const CUtensorMap* map = is_k ? &tma.k : &tma.v;
+          const int z = b * p.Hkv + g;  // which [n_kv][head_dim] matrix of the shard-major copy
+          const int n_stages = is_k ? kKStages : kVStages;
+          const int full0 = is_k ? K_FULL : V_FULL, empty0 = is_k ? K_EMPTY : V_EMPTY;
+          const uint32_t tiles_s = smem_base + (is_k ? kOffK : kOffV);
+          const bool leader = elect_one();
+          for (int i = 0; !w.done(); w.next(), ++i) {
+            // slot of the tile's first key; the box always holds 128 rows (rows past the visible prefix belong to
+            // later keys or, past the end of the matrix, are zero-filled: they are masked either way)
+            const int slot = __ldg(kv_off + w.kk) + w.t0;
+            const int st = i % n_stages;
+            note(8 * i + 1);
+            wait_bar(wc, bar(empty0 + st), (uint32_t)(((i / n_stages) & 1) ^ 1), is_k ? 9 : 10, i);
+            if (leader) {
+              const uint32_t dst = tiles_s + (uint32_t)(st * kTileBytes), fb = bar(full0 + st);
+              mbar_expect_tx(fb, (uint32_t)kTileBytes);
+              tma_tile3(dst, map, 0, slot, z, fb);
+              tma_tile3(dst + kHalfBytes, map, 64, slot, z, fb);
+            }
+            __syncwarp();
             note(8 * i + 2);
-          } else if ((i & 1) == lw - 1) {
-            static_assert(kVStages == 2, "V stage = tile parity = loader warp");
-            const int st = i & 1;
-            note(8 * i + 3);
-            wait_bar(wc, bar(V_EMPTY + st), (uint32_t)(((i / kVStages) & 1) ^ 1), 10, i);
-            gather_rows(smem_base + kOffV + st * kTileBytes, n, lane, tok_of,
-                        [&](int, int tok) { return vb + (int64_t)tok * p.vs.token; });
-            cp_async_wait_all();
-            fence_proxy_async();
-            mbar_arrive(bar(V_FULL + st));
-            note(8 * i + 4);
           }
         }
-        if (lw == 0 && announced >= 0) {
-          cp_async_wait_all();
-          fence_proxy_async();
-          mbar_arrive(bar(K_FULL + announced));
-        }
-        note(8 * i + 7);
       }
-      cp_async_wait_all();
     }
   }
   __syncthreads();
@@ -658,16 +727,112 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(AttnParams p, int 
 
 }  // namespace tc
 
-cudaError_t launch_attn_tc(const AttnParams& p, cudaStream_t stream) {
+namespace {
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// cuTensorMapEncodeTiled through the runtime, so that the library does not link against the driver library.
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      f = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(f);
+  }();
+  return fn;
+}
+
+int64_t gcd64(int64_t a, int64_t b) {
+  while (b) {
+    const int64_t t = a % b;
+    a = b;
+    b = t;
+  }
+  return a;
+}
+
+// The 2-D view [rows][head_dim] of a token-major tensor that the row gather needs: rows lie `pitch` elements apart,
+// pitch = gcd of the strides of the axes that have more than one entry.  Fails if rows would overlap (pitch <
+// head_dim) or the row count does not fit the 32-bit TMA coordinates.
+struct RowView {
+  int64_t pitch = 0, rows = 0;
+  int32_t per_batch = 0, per_token = 0, per_head = 0;
+  bool ok = false;
+};
+RowView row_view(const Strides& st, int64_t batch, int64_t tokens, int64_t heads) {
+  RowView v;
+  int64_t pitch = 0;
+  if (batch > 1) pitch = gcd64(pitch, st.batch);
+  if (tokens > 1) pitch = gcd64(pitch, st.token);
+  if (heads > 1) pitch = gcd64(pitch, st.head);
+  if (pitch == 0) pitch = tc::kD;
+  if (pitch < tc::kD || st.batch < 0 || st.token < 0 || st.head < 0) return v;
+  const int64_t pb = batch > 1 ? st.batch / pitch : 0, pt = tokens > 1 ? st.token / pitch : 0,
+                ph = heads > 1 ? st.head / pitch : 0;
+  const int64_t rows = (batch - 1) * pb + (tokens - 1) * pt + (heads - 1) * ph + 1;
+  if (rows >= (int64_t)1 << 31 || pitch * 2 >= (int64_t)1 << 40) return v;
+  v.pitch = pitch;
+  v.rows = rows;
+  v.per_batch = (int32_t)pb;
+  v.per_token = (int32_t)pt;
+  v.per_head = (int32_t)ph;
+  v.ok = true;
+  return v;
+}
+
+bool encode_rows(CUtensorMap* map, const void* base, const RowView& v) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)tc::kD, (cuuint64_t)v.rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)v.pitch * 2};
+  const cuuint32_t box[2] = {64, 1};  // 128 bytes of one row; tile::gather4 brings four such rows per instruction
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Shard-major K or V copy as a 3-D tensor [batch * kv_heads][n_kv][head_dim]; box = 128 rows x 64 columns.
+bool encode_sorted(CUtensorMap* map, const void* base, int64_t n_kv, int64_t n_mats) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)tc::kD, (cuuint64_t)n_kv, (cuuint64_t)n_mats};
+  const cuuint64_t strides[2] = {(cuuint64_t)tc::kD * 2, (cuuint64_t)n_kv * tc::kD * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)tc::kNMax, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+// Whether the tensor-core kernel can address the queries of this call through a 2-D tensor map.
+bool attn_tc_supports(const AttnParams& p) { return row_view(p.qs, p.batch, p.plan.n_q, p.H).ok; }
+
+cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void* v_sorted, cudaStream_t stream) {
   cudaError_t e = cudaFuncSetAttribute(tc::attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        tc::kSmemBytes);
   if (e != cudaSuccess) return e;
+  const RowView vq = row_view(p.qs, p.batch, p.plan.n_q, p.H);
+  tc::TmaArgs tma;
+  const int64_t n_mats = (int64_t)p.batch * p.Hkv;
+  if (!vq.ok || !encode_rows(&tma.q, p.q, vq) || !encode_sorted(&tma.k, k_sorted, p.plan.n_kv, n_mats) ||
+      !encode_sorted(&tma.v, v_sorted, p.plan.n_kv, n_mats)) {
+    set_error("tensor-core attention: could not describe q/k/v to the TMA unit (strides or driver entry point)");
+    return cudaErrorInvalidValue;
+  }
+  tma.qr = {vq.per_batch, vq.per_token, vq.per_head};
   // stack as many of the G heads of a KV head into one MMA tile as divide G (at most 8)
   int lg = 0;
   while (lg < 3 && p.G % (2 << lg) == 0) ++lg;
   const int n_parts = p.fused ? 1 : p.plan.n_kv_shards;
   dim3 grid(p.plan.n_qtiles[3 - lg], p.H >> lg, p.batch * n_parts);
-  tc::attn_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(p, lg);
+  tc::attn_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(p, lg, tma);
   count_launch();
   return cudaGetLastError();
 }

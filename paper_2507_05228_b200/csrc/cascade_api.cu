@@ -429,9 +429,34 @@ static bool use_tc(const cascade_plan_t* plan, cascade_dtype_t dtype, int d) {
   return dtype == CASCADE_BF16 && d == 128 && plan->dev.n_q > 1;
 }
 
+// Shard-major K and V copies for the tensor-core path: two regions of batch * kv_heads * n_kv rows of 256 bytes.
+static size_t sorted_kv_bytes(const cascade_plan_t* plan, int batch, int Hkv) {
+  return align_up((size_t)batch * Hkv * plan->dev.n_kv * 128 * 2, 256);
+}
+
 static size_t decode_ws_bytes(const cascade_plan_t* plan, cascade_dtype_t dtype, int batch, int H, int d) {
   const size_t rows = (size_t)batch * plan->dev.n_kv_shards * plan->dev.n_q * H;
   return align_up(rows * d * elt_size(dtype), 256) + 2 * align_up(rows * 4, 256);
+}
+
+// Tensor-core route: shard gather of K and V into the workspace, then the attention kernel (two launches).  Falls back
+// to the ALU kernel if the query strides cannot be described to the TMA unit.
+static cascade_status_t run_tc(const AttnParams& p, const char* fn, const cascade_plan_t* plan, void* workspace,
+                               size_t workspace_bytes, cudaStream_t st, cudaError_t* launch_error) {
+  if (!attn_tc_supports(p)) {
+    *launch_error = launch_attn_simt(p, CASCADE_BF16, st);
+    return CASCADE_OK;
+  }
+  const size_t each = sorted_kv_bytes(plan, p.batch, p.Hkv);
+  if (!workspace || workspace_bytes < 2 * each || ((uintptr_t)workspace & 255)) {
+    set_error("%s: workspace of %zu bytes (256-byte aligned) required for the shard-major K/V copies, got %zu", fn,
+              2 * each, workspace_bytes);
+    return CASCADE_ERR_WORKSPACE;
+  }
+  char* ws = (char*)workspace;
+  *launch_error = launch_gather_kv(p, ws, ws + each, st);
+  if (*launch_error == cudaSuccess) *launch_error = launch_attn_tc(p, ws, ws + each, st);
+  return CASCADE_OK;
 }
 
 }  // namespace cascade
@@ -449,12 +474,12 @@ cascade_status_t cascade_workspace_bytes(const cascade_plan_t* plan, int32_t whi
     set_error("cascade_workspace_bytes: bad batch or head counts");
     return CASCADE_ERR_INVALID_ARG;
   }
+  const bool decode = use_decode(plan, dtype, n_heads, n_kv_heads, head_dim);
+  const size_t tc_bytes = !decode && use_tc(plan, dtype, head_dim) ? 2 * sorted_kv_bytes(plan, batch, n_kv_heads) : 0;
   if (which_call == CASCADE_CALL_PARTIALS) {
-    *out_bytes = 0;
+    *out_bytes = tc_bytes;
   } else if (which_call == CASCADE_CALL_SHARDED) {
-    *out_bytes = use_decode(plan, dtype, n_heads, n_kv_heads, head_dim)
-                     ? decode_ws_bytes(plan, dtype, batch, n_heads, head_dim)
-                     : 0;
+    *out_bytes = decode ? decode_ws_bytes(plan, dtype, batch, n_heads, head_dim) : tc_bytes;
   } else {
     set_error("cascade_workspace_bytes: unknown call %d", which_call);
     return CASCADE_ERR_INVALID_ARG;
@@ -468,8 +493,6 @@ cascade_status_t cascade_attn_partials(const cascade_plan_t* plan, cascade_dtype
                                        cascade_strides_t k_strides, const void* v, cascade_strides_t v_strides,
                                        void* o_part, float* m_part, float* l_part, void* workspace,
                                        size_t workspace_bytes, void* stream) {
-  (void)workspace;
-  (void)workspace_bytes;
   cascade_status_t s = check_attn_args("cascade_attn_partials", plan, dtype, batch, n_heads, n_kv_heads,
                                        head_dim, q, q_strides, k, k_strides, v, v_strides);
   if (s != CASCADE_OK) return s;
@@ -489,9 +512,14 @@ cascade_status_t cascade_attn_partials(const cascade_plan_t* plan, cascade_dtype
   p.l_part = l_part;
   cudaStream_t st = (cudaStream_t)stream;
   cudaError_t e;
-  if (use_decode(plan, dtype, n_heads, n_kv_heads, head_dim)) e = launch_decode(p, st);
-  else if (use_tc(plan, dtype, head_dim)) e = launch_attn_tc(p, st);
-  else e = launch_attn_simt(p, dtype, st);
+  if (use_decode(plan, dtype, n_heads, n_kv_heads, head_dim)) {
+    e = launch_decode(p, st);
+  } else if (use_tc(plan, dtype, head_dim)) {
+    cascade_status_t ws = run_tc(p, "cascade_attn_partials", plan, workspace, workspace_bytes, st, &e);
+    if (ws != CASCADE_OK) return ws;
+  } else {
+    e = launch_attn_simt(p, dtype, st);
+  }
   if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_partials: launch");
   return CASCADE_OK;
 }
@@ -597,7 +625,13 @@ cascade_status_t cascade_attn_sharded(const cascade_plan_t* plan, cascade_dtype_
   p.o_out = o_out;
   p.os = {o_strides.batch, o_strides.token, o_strides.head};
   p.lse_out = lse_out;
-  cudaError_t e = use_tc(plan, dtype, head_dim) ? launch_attn_tc(p, st) : launch_attn_simt(p, dtype, st);
+  cudaError_t e;
+  if (use_tc(plan, dtype, head_dim)) {
+    cascade_status_t ws = run_tc(p, "cascade_attn_sharded", plan, workspace, workspace_bytes, st, &e);
+    if (ws != CASCADE_OK) return ws;
+  } else {
+    e = launch_attn_simt(p, dtype, st);
+  }
   if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_sharded: launch");
   return CASCADE_OK;
 }

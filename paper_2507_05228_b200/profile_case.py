@@ -37,11 +37,16 @@ def main():
     o = torch.empty_like(q)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     parts = None
+    ws = None
+    if w.n_q > 1:
+        nb = cb.cascade_workspace_bytes(plan, cb.CALL_SHARDED, cb.BF16 if w.dtype == "bf16" else cb.F32, w.B, w.H, w.Hkv,
+                                        w.d)
+        ws = torch.empty(max(nb, 1), dtype=torch.uint8, device="cuda")
     if args.route in ("partials", "merge", "decode"):
-        parts = cb.cascade_attn_partials(plan, q, k, v, w.scale)
+        parts = cb.cascade_attn_partials(plan, q, k, v, w.scale, workspace=ws)
     fn = {
-        "fused": lambda: cb.cascade_attn_sharded(plan, q, k, v, w.scale, out=o, want_lse=False),
-        "partials": lambda: cb.cascade_attn_partials(plan, q, k, v, w.scale, out=parts),
+        "fused": lambda: cb.cascade_attn_sharded(plan, q, k, v, w.scale, out=o, want_lse=False, workspace=ws),
+        "partials": lambda: cb.cascade_attn_partials(plan, q, k, v, w.scale, out=parts, workspace=ws),
         "decode": lambda: cb.cascade_attn_partials(plan, q, k, v, w.scale, out=parts),
         "merge": lambda: cb.cascade_merge(*parts, plan.dev_ptr("q_idx") if w.n_q > 1 else 0, out=o, want_lse=False),
     }[args.route]
