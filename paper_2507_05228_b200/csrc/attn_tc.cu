@@ -21,14 +21,14 @@
 //         its softmax.  QK_s(i+1) overwrites the columns PV_s(i) reads P from; MMAs execute in issue order, which
 //         makes that safe without a barrier.  The whole warp runs the loop and one elected lane issues, so that
 //         descriptors and addresses stay warp-uniform.
-//   9-11  loaders, all TMA, completion counted in bytes on an mbarrier, data written in the 128-byte-swizzled layout
-//         the MMA descriptors expect.  Warp 9 streams the K tiles and warp 10 the V tiles from the shard-major
-//         copies that the gather pass (gather.cu) wrote: the visible prefix of a shard is a contiguous run of
-//         rows there, so a tile is two 16 KiB box loads.  Warp 11 brings the two query sub-tiles straight from
-//         the caller's tensor with index-mapped row gathers (tile::gather4: four rows of 128 bytes per
-//         instruction); that is done once per CTA only, a row gather being far too slow for the K/V stream
-//         (measured: one 512-byte gather per ~36 cycles per SM; 16-byte cp.async: one 512-byte request per ~90
-//         cycles per warp).
+//   9-10  loaders: TMA box loads, completion counted in bytes on an mbarrier, data written in the 128-byte-swizzled
+//         layout the MMA descriptors expect.  Warp 9 streams the K tiles and warp 10 the V tiles from the
+//         shard-major copies that the gather pass (gather.cu) wrote: the visible prefix of a shard is a
+//         contiguous run of rows there, so a tile is two 16 KiB box loads.  An index-mapped gather straight from
+//         the caller's tensors was far too slow for the K/V stream (measured: one 512-byte TMA row gather per ~36
+//         cycles per SM; 16-byte cp.async: one 512-byte request per ~90 cycles per warp).  The two query
+//         sub-tiles are gathered once per CTA by the softmax threads themselves (plain 16-byte loads).
+//   11    idle (keeps the register-reallocation groups of four warps whole).
 // Every mbarrier wait is bounded: on expiry the CTA raises a flag, records a code in the plan's status word
 // and drains without waiting again.
 #include <cuda.h>
@@ -148,16 +148,6 @@ __device__ __forceinline__ bool wait_bar(const WaitCtx& c, uint32_t bar, uint32_
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// TMA row gather: rows r0..r3 of the 2-D tensor, 64 elements (128 bytes) starting at column `col`, land as four
-// consecutive 128-byte rows at `dst` (swizzled by the hardware according to the shared-memory address).
-__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map, int col, int r0, int r1, int r2,
-                                            int r3, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cta.global.tile::gather4.mbarrier::complete_tx::bytes "
-      "[%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(col), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar)
-      : "memory");
-}
 // TMA box load: 128 rows x 64 elements of the 3-D tensor [matrix z][row y][column x] land as 128 rows of 128 bytes.
 __device__ __forceinline__ void tma_tile3(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
   asm volatile(
@@ -312,14 +302,8 @@ struct TileWalk {
   }
 };
 
-// How a (batch, token, head) triple maps to a row of the 2-D view [rows][head_dim] a row-gather tensor map describes.
-struct RowMap {
-  int32_t per_batch, per_token, per_head;
-};
 struct TmaArgs {
-  CUtensorMap q;     // the caller's query tensor as [rows][head_dim]
   CUtensorMap k, v;  // shard-major copies as [batch * kv_heads][n_kv][head_dim]
-  RowMap qr;
 };
 
 __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_constant__ AttnParams p, int lg,
@@ -375,10 +359,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   };
 
   if (tid == 0) {
-    mbar_init(bar(Q_FULL), 1);  // the *_FULL barriers: one arrival that announces the byte count, then the bytes
-    mbar_init(bar(Q_FULL + 1), 1);
+    mbar_init(bar(Q_FULL), 128);  // every thread of the sub-tile's softmax group brings a share of the rows
+    mbar_init(bar(Q_FULL + 1), 128);
     for (int s = 0; s < kKStages; ++s) {
-      mbar_init(bar(K_FULL + s), 1);
+      mbar_init(bar(K_FULL + s), 1);  // TMA: one arrival that announces the byte count, then the bytes
       mbar_init(bar(K_EMPTY + s), 1);
     }
     for (int s = 0; s < kVStages; ++s) {
@@ -432,6 +416,30 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       int i = 0;  // KV tile counter
       TileWalk w;
       w.start(need_of, k_begin, k_end);
+      if (!w.done()) {
+        // Query sub-tile (row r = slot r / Gp, head r % Gp): this group's 128 threads gather it from the caller's tensor
+        // while they have nothing else to do, 16 bytes per thread and row, half a warp per 256-byte row, into the
+        // 128-byte-swizzled [2][128][128 B] layout.  Rows past the end of the sub-tile repeat its last row (their
+        // results are discarded).
+        const int chunk = m & 15;
+        const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(p.q) + (int64_t)b * p.qs.batch + chunk * 8;
+        uint4 qv[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int r = (m >> 4) + 8 * j;
+          const int tok = __ldg(q_idx + sub_row0 + min(r >> lg, sub_nrows - 1));
+          qv[j] = __ldg(reinterpret_cast<const uint4*>(qb + (int64_t)tok * p.qs.token +
+                                                       (int64_t)(h0 + (r & (Gp - 1))) * p.qs.head));
+        }
+        uint8_t* q_tile = smem + kOffQ + s * kTileBytes + (chunk >> 3) * kHalfBytes;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int r = (m >> 4) + 8 * j;
+          *reinterpret_cast<uint4*>(q_tile + r * 128 + (((chunk & 7) ^ (r & 7)) << 4)) = qv[j];
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> tensor-core reads
+        mbar_arrive(bar(Q_FULL + s));
+      }
       // this row's prefix length in the shard being walked, fetched one shard ahead
       int vis_next = (!w.done() && row_ok) ? __ldg(vis_row + w.kk) : 0;
       for (; !w.done(); w.next(), ++i) {
@@ -664,33 +672,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       // ---------------------------------------------------------------- loaders
       // Every barrier is served by one warp only, in tile order: a phase-parity wait cannot tell "one phase behind"
       // from "one phase ahead", so a warp must never skip a use of a stage.
-      //   warp 9: the K tiles, warp 10: the V tiles, warp 11: the query sub-tiles.
+      //   warp 9: the K tiles, warp 10: the V tiles (warp 11 has no work).
       const int lw = warp - 9;
       TileWalk w;
       w.start(need_of, k_begin, k_end);
       if (!w.done()) {
-        if (lw == 2) {
-          // Query rows: row m of the sub-tile = slot m / Gp, head m % Gp; lane l brings rows 4 l .. 4 l + 3, the two
-          // 128-byte halves of head_dim with one gather each.  Rows past the end of a sub-tile repeat its last
-          // row (their results are discarded), so no out-of-range coordinate is ever used.
-          for (int s = 0; s < n_sub; ++s) {
-            const int sub_row0 = row0 + s * R;
-            const int sub_nrows = min(R, nrows - s * R);
-            int r[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const int m = 4 * lane + j;
-              const int tok = __ldg(q_idx + sub_row0 + min(m >> lg, sub_nrows - 1));
-              r[j] = b * tma.qr.per_batch + tok * tma.qr.per_token + (h0 + (m & (Gp - 1))) * tma.qr.per_head;
-            }
-            const uint32_t fb = bar(Q_FULL + s);
-            if (lane == 0) mbar_expect_tx(fb, (uint32_t)kTileBytes);
-            __syncwarp();
-            const uint32_t dst = smem_base + kOffQ + (uint32_t)(s * kTileBytes + 4 * lane * 128);
-            tma_gather4(dst, &tma.q, 0, r[0], r[1], r[2], r[3], fb);
-            tma_gather4(dst + kHalfBytes, &tma.q, 64, r[0], r[1], r[2], r[3], fb);
-          }
-        } else {
+        if (lw < 2) {
           const bool is_k = lw == 0;
           const CUtensorMap* map = is_k ? &tma.k : &tma.v;
           const int z = b * p.Hkv + g;  // which [n_kv][head_dim] matrix of the shard-major copy
@@ -746,56 +733,6 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-int64_t gcd64(int64_t a, int64_t b) {
-  while (b) {
-    const int64_t t = a % b;
-    a = b;
-    b = t;
-  }
-  return a;
-}
-
-// The 2-D view [rows][head_dim] of a token-major tensor that the row gather needs: rows lie `pitch` elements apart,
-// pitch = gcd of the strides of the axes that have more than one entry.  Fails if rows would overlap (pitch <
-// head_dim) or the row count does not fit the 32-bit TMA coordinates.
-struct RowView {
-  int64_t pitch = 0, rows = 0;
-  int32_t per_batch = 0, per_token = 0, per_head = 0;
-  bool ok = false;
-};
-RowView row_view(const Strides& st, int64_t batch, int64_t tokens, int64_t heads) {
-  RowView v;
-  int64_t pitch = 0;
-  if (batch > 1) pitch = gcd64(pitch, st.batch);
-  if (tokens > 1) pitch = gcd64(pitch, st.token);
-  if (heads > 1) pitch = gcd64(pitch, st.head);
-  if (pitch == 0) pitch = tc::kD;
-  if (pitch < tc::kD || st.batch < 0 || st.token < 0 || st.head < 0) return v;
-  const int64_t pb = batch > 1 ? st.batch / pitch : 0, pt = tokens > 1 ? st.token / pitch : 0,
-                ph = heads > 1 ? st.head / pitch : 0;
-  const int64_t rows = (batch - 1) * pb + (tokens - 1) * pt + (heads - 1) * ph + 1;
-  if (rows >= (int64_t)1 << 31 || pitch * 2 >= (int64_t)1 << 40) return v;
-  v.pitch = pitch;
-  v.rows = rows;
-  v.per_batch = (int32_t)pb;
-  v.per_token = (int32_t)pt;
-  v.per_head = (int32_t)ph;
-  v.ok = true;
-  return v;
-}
-
-bool encode_rows(CUtensorMap* map, const void* base, const RowView& v) {
-  EncodeTiledFn fn = encode_tiled_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[2] = {(cuuint64_t)tc::kD, (cuuint64_t)v.rows};
-  const cuuint64_t strides[1] = {(cuuint64_t)v.pitch * 2};
-  const cuuint32_t box[2] = {64, 1};  // 128 bytes of one row; tile::gather4 brings four such rows per instruction
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // Shard-major K or V copy as a 3-D tensor [batch * kv_heads][n_kv][head_dim]; box = 128 rows x 64 columns.
 bool encode_sorted(CUtensorMap* map, const void* base, int64_t n_kv, int64_t n_mats) {
   EncodeTiledFn fn = encode_tiled_fn();
@@ -811,22 +748,16 @@ bool encode_sorted(CUtensorMap* map, const void* base, int64_t n_kv, int64_t n_m
 
 }  // namespace
 
-// Whether the tensor-core kernel can address the queries of this call through a 2-D tensor map.
-bool attn_tc_supports(const AttnParams& p) { return row_view(p.qs, p.batch, p.plan.n_q, p.H).ok; }
-
 cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void* v_sorted, cudaStream_t stream) {
   cudaError_t e = cudaFuncSetAttribute(tc::attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        tc::kSmemBytes);
   if (e != cudaSuccess) return e;
-  const RowView vq = row_view(p.qs, p.batch, p.plan.n_q, p.H);
   tc::TmaArgs tma;
   const int64_t n_mats = (int64_t)p.batch * p.Hkv;
-  if (!vq.ok || !encode_rows(&tma.q, p.q, vq) || !encode_sorted(&tma.k, k_sorted, p.plan.n_kv, n_mats) ||
-      !encode_sorted(&tma.v, v_sorted, p.plan.n_kv, n_mats)) {
-    set_error("tensor-core attention: could not describe q/k/v to the TMA unit (strides or driver entry point)");
+  if (!encode_sorted(&tma.k, k_sorted, p.plan.n_kv, n_mats) || !encode_sorted(&tma.v, v_sorted, p.plan.n_kv, n_mats)) {
+    set_error("tensor-core attention: could not build the TMA descriptors of the shard-major K/V copies");
     return cudaErrorInvalidValue;
   }
-  tma.qr = {vq.per_batch, vq.per_token, vq.per_head};
   // stack as many of the G heads of a KV head into one MMA tile as divide G (at most 8)
   int lg = 0;
   while (lg < 3 && p.G % (2 << lg) == 0) ++lg;

@@ -439,14 +439,9 @@ static size_t decode_ws_bytes(const cascade_plan_t* plan, cascade_dtype_t dtype,
   return align_up(rows * d * elt_size(dtype), 256) + 2 * align_up(rows * 4, 256);
 }
 
-// Tensor-core route: shard gather of K and V into the workspace, then the attention kernel (two launches).  Falls back
-// to the ALU kernel if the query strides cannot be described to the TMA unit.
+// Tensor-core route: shard gather of K and V into the workspace, then the attention kernel (two launches).
 static cascade_status_t run_tc(const AttnParams& p, const char* fn, const cascade_plan_t* plan, void* workspace,
                                size_t workspace_bytes, cudaStream_t st, cudaError_t* launch_error) {
-  if (!attn_tc_supports(p)) {
-    *launch_error = launch_attn_simt(p, CASCADE_BF16, st);
-    return CASCADE_OK;
-  }
   const size_t each = sorted_kv_bytes(plan, p.batch, p.Hkv);
   if (!workspace || workspace_bytes < 2 * each || ((uintptr_t)workspace & 255)) {
     set_error("%s: workspace of %zu bytes (256-byte aligned) required for the shard-major K/V copies, got %zu", fn,

@@ -87,7 +87,6 @@ cudaError_t launch_attn_simt(const AttnParams& p, cascade_dtype_t dtype, cudaStr
 // k_sorted / v_sorted: the shard-major copies written by launch_gather_kv, [batch][kv_head][n_kv][128] bf16
 cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void* v_sorted, cudaStream_t stream);
 cudaError_t launch_gather_kv(const AttnParams& p, void* k_out, void* v_out, cudaStream_t stream);
-bool attn_tc_supports(const AttnParams& p);  // the q strides can be described to the TMA unit
 cudaError_t launch_decode(const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_merge(const MergeParams& p, cascade_dtype_t dtype, cudaStream_t stream);
 
