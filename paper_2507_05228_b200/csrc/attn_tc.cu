@@ -8,8 +8,10 @@
 // One CTA owns two such sub-tiles (the next 128 / Gp slots of the same shard, same heads), which share every K/V
 // tile, and either one KV shard (partials: Algorithm 3 for the pair) or all KV shards one after another (fused:
 // the carry n, w, o of Algorithm 4 is the running max / sum / output of the streaming softmax).
-// Each shard's visible prefix is walked in tiles of at most 128 keys; the last tile of a prefix is narrowed to a
-// multiple of 32 keys.
+// The KV shards are walked one after another; each shard's visible prefix (as seen by the CTA's last row, which has
+// the longest one) is cut into chunks of 32 keys, and four consecutive chunks of that stream - possibly from
+// different shards - form one MMA tile of 128 keys, so that only the last tile of a CTA is narrower.  (An MMA costs
+// the same for 32 keys as for 128, and every tile costs one softmax round trip.)
 //
 // Warp roles (12 warps):
 //   0-3   softmax of sub-tile 0, 4-7 softmax of sub-tile 1: thread = MMA row = TMEM lane.  Reads the logits S with
@@ -50,7 +52,9 @@ constexpr uint32_t kTmemCols = 512;       // S0 | S1 | O0 | O1, 128 columns each
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 constexpr int kRegsSoftmax = 216;
 constexpr int kRegsOther = 72;
-constexpr int kMaxShardsInSmem = 96;      // per-shard prefix lengths are staged in shared memory up to this many
+constexpr int kChunk = 32;                // keys per chunk of the KV stream
+constexpr int kChunkBytes = kChunk * 128; // one 64-column half of a chunk in a tile
+constexpr int kMaxShards = 88;            // KV shards per CTA whose bookkeeping fits in shared memory
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int kOffQ = 0;
@@ -59,8 +63,8 @@ constexpr int kOffV = kOffK + kKStages * kTileBytes;
 constexpr int kOffBar = kOffV + kVStages * kTileBytes;
 constexpr int kNumBars = 24;
 constexpr int kOffMisc = kOffBar + kNumBars * 8;   // tmem slot, abort flag, 12 progress words
-constexpr int kOffShard = kOffMisc + 64;           // int32 [3][kMaxShardsInSmem]: need, first row of sub-tile 0 / 1
-constexpr int kSmemBytes = kOffShard + 3 * kMaxShardsInSmem * 4 + 1024;  // + alignment slack
+constexpr int kOffShard = kOffMisc + 64;           // int32 [5][kMaxShards], see ShardTab
+constexpr int kSmemBytes = kOffShard + 5 * kMaxShards * 4 + 1024;  // + alignment slack
 static_assert(kSmemBytes <= 232448, "exceeds the 227 KiB a CTA may use");
 
 enum Bar {
@@ -148,7 +152,7 @@ __device__ __forceinline__ bool wait_bar(const WaitCtx& c, uint32_t bar, uint32_
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// TMA box load: 128 rows x 64 elements of the 3-D tensor [matrix z][row y][column x] land as 128 rows of 128 bytes.
+// TMA box load: 32 rows x 64 elements of the 3-D tensor [matrix z][row y][column x] land as 32 rows of 128 bytes.
 __device__ __forceinline__ void tma_tile3(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
@@ -270,35 +274,28 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-// The CTA's sequence of KV tiles: shard by shard, each shard's visible prefix (as seen by the CTA's last row, which
-// has the longest one) in pieces of at most 128 keys.  Every role walks the same sequence.
-struct TileWalk {
-  const int32_t* need_of;  // vis[last row of the CTA][*] (shared-memory copy when it fits)
-  int k_end, kk, t0, need;
-  __device__ __forceinline__ void seek() {
-    t0 = 0;
-    need = 0;
-    while (kk < k_end) {
-      need = need_of[kk];
-      if (need > 0) break;
-      ++kk;
-    }
+// Bookkeeping of the shards of which the CTA sees anything ("active" shards, in walk order), in shared memory.
+struct ShardTab {
+  int32_t need[kMaxShards];    // visible prefix of the CTA's last row = keys of the shard that are walked
+  int32_t first[2][kMaxShards];  // visible prefix of the first row of sub-tile 0 / 1: chunks below it need no mask
+  int32_t slot0[kMaxShards];   // position of the shard's first key in the shard-major K/V copies
+  int32_t kk[kMaxShards];      // shard id
+};
+// Cursor over the chunk stream: chunk c of active shard j.
+struct ChunkCursor {
+  int j, c, nc;  // nc = chunks of shard j
+  __device__ __forceinline__ void start(const ShardTab* t, int n_act) {
+    j = 0;
+    c = 0;
+    nc = n_act > 0 ? (t->need[0] + kChunk - 1) / kChunk : 0;
   }
-  __device__ __forceinline__ void start(const int32_t* need_of_, int k_begin, int k_end_) {
-    need_of = need_of_;
-    k_end = k_end_;
-    kk = k_begin;
-    seek();
-  }
-  __device__ __forceinline__ bool done() const { return kk >= k_end; }
-  __device__ __forceinline__ int keys() const { return min(kNMax, need - t0); }  // real keys in this tile
-  __device__ __forceinline__ int n() const { return (keys() + 31) & ~31; }       // MMA width: multiple of 32
-  __device__ __forceinline__ void next() {
-    t0 += kNMax;
-    if (t0 >= need) {
-      ++kk;
-      seek();
-    }
+  // moves to the next chunk; returns true if that entered a new shard
+  __device__ __forceinline__ bool advance(const ShardTab* t, int n_act) {
+    if (++c < nc) return false;
+    ++j;
+    c = 0;
+    nc = j < n_act ? (t->need[j] + kChunk - 1) / kChunk : 0;
+    return true;
   }
 };
 
@@ -316,7 +313,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kOffMisc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffMisc + 4);
   volatile int* progress = reinterpret_cast<volatile int*>(smem + kOffMisc + 8);  // [12]
-  int32_t* shard_tab = reinterpret_cast<int32_t*>(smem + kOffShard);              // [3][kMaxShardsInSmem]
+  ShardTab* tab = reinterpret_cast<ShardTab*>(smem + kOffShard);
+  volatile int* stream_info = reinterpret_cast<volatile int*>(smem + kOffMisc + 56);  // [0] active shards, [1] chunks
 
   // lg = log2(Gp): Gp heads stacked per tile, R = 128 / Gp slots per sub-tile, 2 R slots per CTA
   const int Gp = 1 << lg, R = kM >> lg;
@@ -339,19 +337,35 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   const int32_t* kv_off = pl.kv_off + (size_t)map * (P + 1);
   const int32_t* vis = pl.vis + (size_t)map * pl.n_q * P;
   const int k_begin = p.fused ? 0 : part, k_end = p.fused ? P : part + 1;
-  // Per-shard prefix lengths the roles consult at every shard change: the CTA's last row (longest prefix, drives the
-  // tile walk) and the first row of each sub-tile (shortest prefix, decides whether a tile needs the mask).
-  const int32_t* need_of = vis + (size_t)(row0 + nrows - 1) * P;
-  const int32_t* first_of[2] = {vis + (size_t)row0 * P, vis + (size_t)(row0 + (n_sub - 1) * R) * P};
-  if (P <= kMaxShardsInSmem) {
-    for (int kk = tid; kk < P; kk += kThreads) {
-      shard_tab[kk] = __ldg(need_of + kk);
-      shard_tab[kMaxShardsInSmem + kk] = __ldg(first_of[0] + kk);
-      shard_tab[2 * kMaxShardsInSmem + kk] = __ldg(first_of[1] + kk);
+  if (warp == 0) {
+    // Compact the shards of which the CTA's last row (longest prefix; rows ascend) sees something, with what the
+    // roles need per shard, and count the chunks of the stream.
+    const int32_t* need_of = vis + (size_t)(row0 + nrows - 1) * P;
+    const int32_t* first0 = vis + (size_t)row0 * P;
+    const int32_t* first1 = vis + (size_t)(row0 + (n_sub - 1) * R) * P;
+    int n_act = 0, n_chunks = 0;
+    for (int base = k_begin; base < k_end; base += 32) {
+      const int kk = base + lane;
+      const int nd = kk < k_end ? __ldg(need_of + kk) : 0;
+      const uint32_t act = __ballot_sync(0xffffffffu, nd > 0);
+      if (nd > 0) {
+        const int pos = n_act + __popc(act & ((1u << lane) - 1u));
+        tab->need[pos] = nd;
+        tab->first[0][pos] = __ldg(first0 + kk);
+        tab->first[1][pos] = __ldg(first1 + kk);
+        tab->slot0[pos] = __ldg(kv_off + kk);
+        tab->kk[pos] = kk;
+      }
+      n_act += __popc(act);
+      int ch = (nd + kChunk - 1) / kChunk;
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) ch += __shfl_xor_sync(0xffffffffu, ch, off);
+      n_chunks += ch;
     }
-    need_of = shard_tab;
-    first_of[0] = shard_tab + kMaxShardsInSmem;
-    first_of[1] = shard_tab + 2 * kMaxShardsInSmem;
+    if (lane == 0) {
+      stream_info[0] = n_act;
+      stream_info[1] = n_chunks;
+    }
   }
   WaitCtx wc{abort_flag, progress, pl.status};
   auto note = [&](int v) {
@@ -389,6 +403,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  const int n_act = stream_info[0];                 // shards of which the CTA sees something
+  const int n_chunks = stream_info[1];              // chunks of the KV stream
+  const int n_tiles = (n_chunks + 3) >> 2;          // MMA tiles: four chunks each, the last one possibly fewer
+  auto tile_chunks = [&](int i) { return min(4, n_chunks - 4 * i); };
 
   if (warp < 8) {
     // ------------------------------------------------------------------ softmax + epilogue
@@ -403,7 +421,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       const int slot = sub_row0 + (row_ok ? slot_local : 0);
       const int head = h0 + (m & (Gp - 1));
       const int32_t* vis_row = vis + (size_t)slot * P;
-      const int32_t* vis_first = first_of[s];  // shortest prefix of the sub-tile
+      const int32_t* vis_first = tab->first[s];  // shortest prefix of the sub-tile, per active shard
       const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
       const uint32_t s_addr = lane_base + (uint32_t)(s * 128);
       const uint32_t o_addr = lane_base + 256u + (uint32_t)(s * 128);
@@ -412,11 +430,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       float m_run = -INFINITY;   // reference max the accumulators are scaled by (may lag by < 2^8)
       float m_true = -INFINITY;  // exact running max
       float l_run = 0.f;
-      int my_vis = 0, full_upto = 0;
-      int i = 0;  // KV tile counter
-      TileWalk w;
-      w.start(need_of, k_begin, k_end);
-      if (!w.done()) {
+      if (n_tiles > 0) {
         // Query sub-tile (row r = slot r / Gp, head r % Gp): this group's 128 threads gather it from the caller's tensor
         // while they have nothing else to do, 16 bytes per thread and row, half a warp per 256-byte row, into the
         // 128-byte-swizzled [2][128][128 B] layout.  Rows past the end of the sub-tile repeat its last row (their
@@ -440,19 +454,36 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> tensor-core reads
         mbar_arrive(bar(Q_FULL + s));
       }
-      // this row's prefix length in the shard being walked, fetched one shard ahead
-      int vis_next = (!w.done() && row_ok) ? __ldg(vis_row + w.kk) : 0;
-      for (; !w.done(); w.next(), ++i) {
-        if (w.t0 == 0) {  // entered a new shard
-          my_vis = vis_next;
-          full_upto = vis_first[w.kk];
-          TileWalk peek = w;  // the next shard with something visible
-          ++peek.kk;
-          peek.seek();
-          vis_next = (!peek.done() && row_ok) ? __ldg(vis_row + peek.kk) : 0;
+      // This row's prefix lengths in the current and the next three active shards (a tile spans at most four), fetched
+      // as the stream moves on so that the loads are off the critical path.
+      auto row_vis = [&](int j) { return (j < n_act && row_ok) ? __ldg(vis_row + tab->kk[j]) : 0; };
+      int vq0 = row_vis(0), vq1 = row_vis(1), vq2 = row_vis(2), vq3 = row_vis(3);
+      ChunkCursor cur;
+      cur.start(tab, n_act);
+      for (int i = 0; i < n_tiles; ++i) {
+        const int nch = tile_chunks(i);
+        // Mask bookkeeping for the tile's four chunks, done before the wait so that it costs nothing: a chunk of shard
+        // j starting at key t0 needs the mask only if it reaches past the shortest prefix of the sub-tile; this row
+        // then sees its first lc = vis - t0 columns.  Chunks a narrow last tile does not have count as fully masked.
+        int lc[4];
+        uint32_t needm = 0;
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          if (ch < nch) {  // warp-uniform
+            const int t0 = cur.c * kChunk;
+            if (t0 + kChunk > vis_first[cur.j]) needm |= 1u << ch;
+            lc[ch] = vq0 - t0;
+            if (cur.advance(tab, n_act)) {
+              vq0 = vq1;
+              vq1 = vq2;
+              vq2 = vq3;
+              vq3 = row_vis(cur.j + 3);
+            }
+          } else {
+            needm |= 1u << ch;
+            lc[ch] = 0;
+          }
         }
-        const int n = w.n();
-        const int nch = n >> 5;
         note(8 * i + 1);
         wait_bar(wc, bar(S_FULL + s), (uint32_t)(i & 1), 1, i);
         tc_fence_after();
@@ -462,18 +493,16 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         if (nch > 2) CASCADE_TMEM_LD32(s_addr + 64, sr, 64);
         if (nch > 3) CASCADE_TMEM_LD32(s_addr + 96, sr, 96);
         tmem_wait_ld();
-        // mask: only tiles that reach past the shortest prefix of the sub-tile need it.  Columns [0, lim) are visible
-        // to this row (lim <= keys <= n, so this also covers columns that were never loaded).  The mask is applied
-        // through a per-chunk bit mask so that the compiler can move several bits at a time into predicates.
-        if (!(n == kNMax && w.t0 + n <= full_upto)) {
-          const int lim = my_vis - w.t0;
+        // The mask is applied through a bit mask so that the compiler can move several bits at a time into predicates.
+        if (needm != 0) {  // warp-uniform
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
-            const int lc = lim - 32 * ch;
-            const uint32_t mk = lc >= 32 ? 0xffffffffu : (lc <= 0 ? 0u : ((1u << lc) - 1u));
+            if ((needm >> ch) & 1u) {  // warp-uniform
+              const uint32_t mk = lc[ch] >= 32 ? 0xffffffffu : (lc[ch] <= 0 ? 0u : ((1u << lc[ch]) - 1u));
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (!((mk >> j) & 1u)) sr[32 * ch + j] = 0xff800000u;  // -inf
+              for (int j = 0; j < 32; ++j)
+                if (!((mk >> j) & 1u)) sr[32 * ch + j] = 0xff800000u;  // -inf
+            }
           }
         }
         float mx[4];
@@ -535,8 +564,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         mbar_arrive(bar(P_FULL + s));
         note(8 * i + 2);
       }
-      const int n_tiles = i;
-      note(8 * i + 3);
+      note(8 * n_tiles + 3);
       // ---- epilogue
       float o_scale = 0.f, m_out = -INFINITY, l_out = 0.f;
       if (n_tiles > 0) {
@@ -600,9 +628,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       const uint32_t q_lo0 = desc_lo(smem_base + kOffQ, 16);
       const uint32_t k_lo0 = desc_lo(smem_base + kOffK, 16);
       const uint32_t v_lo0 = desc_lo(smem_base + kOffV, kHalfBytes);  // the two 64-column halves of d
-      TileWalk w;
-      w.start(need_of, k_begin, k_end);
-      if (!w.done()) {
+      if (n_tiles > 0) {
         auto issue_qk = [&](int s, int i, int n) {  // S_s = Q_s K(i)^T, n keys wide
           const uint32_t q_lo = q_lo0 + (uint32_t)(s * (kTileBytes >> 4));
           const uint32_t k_lo = k_lo0 + (uint32_t)((i % kKStages) * (kTileBytes >> 4));
@@ -630,18 +656,17 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
             }
           }
         };
-        int n_cur = w.n();
         wait_bar(wc, bar(K_FULL), 0u, 7);
         for (int s = 0; s < n_sub; ++s) {
           wait_bar(wc, bar(Q_FULL + s), 0u, 6);
           tc_fence_after();
-          issue_qk(s, 0, n_cur);
+          issue_qk(s, 0, kChunk * tile_chunks(0));
         }
         if (leader) mma_commit(bar(K_EMPTY));
-        w.next();
-        for (int i = 0;; ++i) {
-          const bool has_next = !w.done();
-          const int n_next = has_next ? w.n() : 0;
+        for (int i = 0; i < n_tiles; ++i) {
+          const bool has_next = i + 1 < n_tiles;
+          const int n_cur = kChunk * tile_chunks(i);
+          const int n_next = has_next ? kChunk * tile_chunks(i + 1) : 0;
           note(8 * i + 1);
           wait_bar(wc, bar(V_FULL + i % kVStages), (uint32_t)((i / kVStages) & 1), 4, i);
           for (int s = 0; s < n_sub; ++s) {
@@ -660,9 +685,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
               if (s == n_sub - 1 && leader) mma_commit(bar(K_EMPTY + (i + 1) % kKStages));
             }
           }
-          if (!has_next) break;
-          n_cur = n_next;
-          w.next();
         }
         if (leader) mma_commit(bar(O_FULL));
         note(7);
@@ -674,33 +696,35 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       // from "one phase ahead", so a warp must never skip a use of a stage.
       //   warp 9: the K tiles, warp 10: the V tiles (warp 11 has no work).
       const int lw = warp - 9;
-      TileWalk w;
-      w.start(need_of, k_begin, k_end);
-      if (!w.done()) {
-        if (lw < 2) {
-          const bool is_k = lw == 0;
-          const CUtensorMap* map = is_k ? &tma.k : &tma.v;
-          const int z = b * p.Hkv + g;  // which [n_kv][head_dim] matrix of the shard-major copy
-          const int n_stages = is_k ? kKStages : kVStages;
-          const int full0 = is_k ? K_FULL : V_FULL, empty0 = is_k ? K_EMPTY : V_EMPTY;
-          const uint32_t tiles_s = smem_base + (is_k ? kOffK : kOffV);
-          const bool leader = elect_one();
-          for (int i = 0; !w.done(); w.next(), ++i) {
-            // slot of the tile's first key; the box always holds 128 rows (rows past the visible prefix belong to
-            // later keys or, past the end of the matrix, are zero-filled: they are masked either way)
-            const int slot = __ldg(kv_off + w.kk) + w.t0;
-            const int st = i % n_stages;
-            note(8 * i + 1);
-            wait_bar(wc, bar(empty0 + st), (uint32_t)(((i / n_stages) & 1) ^ 1), is_k ? 9 : 10, i);
+      if (n_tiles > 0 && lw < 2) {
+        const bool is_k = lw == 0;
+        const CUtensorMap* map = is_k ? &tma.k : &tma.v;
+        const int z = b * p.Hkv + g;  // which [n_kv][head_dim] matrix of the shard-major copy
+        const int n_stages = is_k ? kKStages : kVStages;
+        const int full0 = is_k ? K_FULL : V_FULL, empty0 = is_k ? K_EMPTY : V_EMPTY;
+        const uint32_t tiles_s = smem_base + (is_k ? kOffK : kOffV);
+        const bool leader = elect_one();
+        ChunkCursor cur;
+        cur.start(tab, n_act);
+        for (int i = 0; i < n_tiles; ++i) {
+          const int nch = tile_chunks(i);
+          const int st = i % n_stages;
+          note(8 * i + 1);
+          wait_bar(wc, bar(empty0 + st), (uint32_t)(((i / n_stages) & 1) ^ 1), is_k ? 9 : 10, i);
+          const uint32_t dst = tiles_s + (uint32_t)(st * kTileBytes), fb = bar(full0 + st);
+          if (leader) mbar_expect_tx(fb, (uint32_t)(nch * 2 * kChunkBytes));
+          for (int ch = 0; ch < nch; ++ch) {
+            // A chunk is 32 consecutive rows of the shard-major copy.  Rows past the shard's visible prefix belong
+            // to later keys or, past the end of the matrix, are zero-filled: they are masked either way.
+            const int slot = tab->slot0[cur.j] + cur.c * kChunk;
             if (leader) {
-              const uint32_t dst = tiles_s + (uint32_t)(st * kTileBytes), fb = bar(full0 + st);
-              mbar_expect_tx(fb, (uint32_t)kTileBytes);
-              tma_tile3(dst, map, 0, slot, z, fb);
-              tma_tile3(dst + kHalfBytes, map, 64, slot, z, fb);
+              tma_tile3(dst + (uint32_t)(ch * kChunkBytes), map, 0, slot, z, fb);
+              tma_tile3(dst + (uint32_t)(kHalfBytes + ch * kChunkBytes), map, 64, slot, z, fb);
             }
-            __syncwarp();
-            note(8 * i + 2);
+            cur.advance(tab, n_act);
           }
+          __syncwarp();
+          note(8 * i + 2);
         }
       }
     }
@@ -733,13 +757,13 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// Shard-major K or V copy as a 3-D tensor [batch * kv_heads][n_kv][head_dim]; box = 128 rows x 64 columns.
+// Shard-major K or V copy as a 3-D tensor [batch * kv_heads][n_kv][head_dim]; box = one chunk (32 rows) x 64 columns.
 bool encode_sorted(CUtensorMap* map, const void* base, int64_t n_kv, int64_t n_mats) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   const cuuint64_t dims[3] = {(cuuint64_t)tc::kD, (cuuint64_t)n_kv, (cuuint64_t)n_mats};
   const cuuint64_t strides[2] = {(cuuint64_t)tc::kD * 2, (cuuint64_t)n_kv * tc::kD * 2};
-  const cuuint32_t box[3] = {64, (cuuint32_t)tc::kNMax, 1};
+  const cuuint32_t box[3] = {64, (cuuint32_t)tc::kChunk, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
