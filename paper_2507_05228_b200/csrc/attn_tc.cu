@@ -304,6 +304,7 @@ struct TmaArgs {
 };
 
 __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_constant__ AttnParams p, int lg,
+                                                              int tile_major,
                                                               const __grid_constant__ TmaArgs tma) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -321,13 +322,32 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   const PlanDev& pl = p.plan;
   const int P = pl.n_kv_shards;
   const int n_parts = p.fused ? 1 : P;
-  const int b = blockIdx.z / n_parts;
-  const int part = blockIdx.z % n_parts;
+  // CTA index -> (query tile, batch, part, head group).  The tile lists are sorted by decreasing work.  With few CTAs
+  // per SM the query tile is the slowest index, so that the heaviest CTAs of all heads and sequences start first and
+  // the light ones fill the tail.  For a large problem the head group is slowest instead: the CTAs running at any
+  // time then read the K/V of few KV heads, which keeps that stream in L2.
+  const int n_hg = p.H >> lg;
+  const int n_qt = pl.n_qtiles[3 - lg];
+  int tile_idx, hg, bz;
+  if (tile_major) {
+    const int per_tile = n_hg * p.batch * n_parts;
+    const int rem = blockIdx.x % per_tile;
+    tile_idx = blockIdx.x / per_tile;
+    hg = rem % n_hg;
+    bz = rem / n_hg;
+  } else {
+    const int rem = blockIdx.x / n_qt;
+    tile_idx = blockIdx.x % n_qt;
+    hg = rem % n_hg;
+    bz = rem / n_hg;
+  }
+  const int b = bz / n_parts;
+  const int part = bz % n_parts;
   const int map = pl.n_maps == 1 ? 0 : b;
-  const int h0 = blockIdx.y * Gp;  // first of the Gp stacked heads
-  const int g = h0 / p.G;          // their KV head
-  const int ts = 3 - lg;           // tile list of 2 R = 256 >> lg slots
-  const int4 qt = pl.qtiles[ts][(size_t)map * pl.n_qtiles[ts] + blockIdx.x];
+  const int h0 = hg * Gp;  // first of the Gp stacked heads
+  const int g = h0 / p.G;  // their KV head
+  const int ts = 3 - lg;   // tile list of 2 R = 256 >> lg slots
+  const int4 qt = pl.qtiles[ts][(size_t)map * pl.n_qtiles[ts] + tile_idx];
   const int row0 = qt.x, nrows = qt.y;
   if (nrows == 0) return;  // padding entry (uniform for the CTA)
   if (*reinterpret_cast<volatile int32_t*>(pl.status) != 0) return;  // an earlier CTA gave up: do not pile on
@@ -786,8 +806,10 @@ cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void
   int lg = 0;
   while (lg < 3 && p.G % (2 << lg) == 0) ++lg;
   const int n_parts = p.fused ? 1 : p.plan.n_kv_shards;
-  dim3 grid(p.plan.n_qtiles[3 - lg], p.H >> lg, p.batch * n_parts);
-  tc::attn_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(p, lg, tma);
+  const int64_t n_ctas = (int64_t)p.plan.n_qtiles[3 - lg] * (p.H >> lg) * p.batch * n_parts;
+  if (n_ctas >= (int64_t)1 << 31) return cudaErrorInvalidConfiguration;
+  const int tile_major = n_ctas <= 8 * 148;  // few CTAs per SM: balance matters more than L2 locality
+  tc::attn_tc_kernel<<<(unsigned)n_ctas, tc::kThreads, tc::kSmemBytes, stream>>>(p, lg, tile_major, tma);
   count_launch();
   return cudaGetLastError();
 }
