@@ -544,22 +544,32 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
         const uint64_t neg_m2 = pack2(neg_m, neg_m);
         uint64_t psum2 = pack2(0.f, 0.f);
+        auto exp_chunk = [&](int ch) {
+          uint32_t pk[16];
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          if (ch < nch) {  // warp-uniform
-            uint32_t pk[16];
-#pragma unroll
-            for (int j = 0; j < 32; j += 2) {
-              float x0, x1;
-              unpack2(ffma2(pack2(__uint_as_float(sr[32 * ch + j]), __uint_as_float(sr[32 * ch + j + 1])), c2, neg_m2),
-                      x0, x1);
-              const float p0 = ex2(x0), p1 = ex2(x1);
-              psum2 = fadd2(psum2, pack2(p0, p1));
-              pk[j >> 1] = pack_bf16x2(p0, p1);
-            }
-            // P as the A operand of the PV product: lane = row, column kk holds keys 2 kk and 2 kk + 1
-            CASCADE_TMEM_ST16(s_addr + (uint32_t)(16 * ch), pk);
+          for (int j = 0; j < 32; j += 2) {
+            float x0, x1;
+            unpack2(ffma2(pack2(__uint_as_float(sr[32 * ch + j]), __uint_as_float(sr[32 * ch + j + 1])), c2, neg_m2), x0,
+                    x1);
+            const float p0 = ex2(x0), p1 = ex2(x1);
+            psum2 = fadd2(psum2, pack2(p0, p1));
+            pk[j >> 1] = pack_bf16x2(p0, p1);
           }
+          // P as the A operand of the PV product: lane = row, column kk holds keys 2 kk and 2 kk + 1
+          CASCADE_TMEM_ST16(s_addr + (uint32_t)(16 * ch), pk);
+        };
+        if (nch == 4) {
+          // The full tile is one straight-line block, so that the scheduler can run the MUFU instructions of one chunk
+          // (8 issue cycles each) under the FMA / convert / store work of its neighbours; with a branch per chunk the
+          // two parts ran back to back (1600 cycles per tile instead of the ~1130 the MUFU unit needs).
+          exp_chunk(0);
+          exp_chunk(1);
+          exp_chunk(2);
+          exp_chunk(3);
+        } else {
+#pragma unroll
+          for (int ch = 0; ch < 3; ++ch)
+            if (ch < nch) exp_chunk(ch);  // warp-uniform
         }
         float psum0, psum1;
         unpack2(psum2, psum0, psum1);
