@@ -46,7 +46,7 @@ constexpr int kNMax = 128;               // keys per KV tile (upper bound)
 constexpr int kD = 128;                  // head_dim
 constexpr int kTileBytes = kM * kD * 2;  // 32 KiB, laid out [2 halves][128 rows][128 bytes]
 constexpr int kHalfBytes = kTileBytes / 2;
-constexpr int kKStages = 3;
+constexpr int kKStages = 2;  // (a third stage bought nothing)
 constexpr int kVStages = 2;
 constexpr uint32_t kTmemCols = 512;       // S0 | S1 | O0 | O1, 128 columns each; P_s aliases the start of S_s
 constexpr float kRescaleThreshold = 8.f;  // log2 units
@@ -54,7 +54,7 @@ constexpr int kRegsSoftmax = 216;
 constexpr int kRegsOther = 72;
 constexpr int kChunk = 32;                // keys per chunk of the KV stream
 constexpr int kChunkBytes = kChunk * 128; // one 64-column half of a chunk in a tile
-constexpr int kMaxShards = 88;            // KV shards per CTA whose bookkeeping fits in shared memory
+constexpr int kMaxShards = 256;           // KV shards per CTA whose bookkeeping fits in shared memory
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int kOffQ = 0;
@@ -269,6 +269,12 @@ __device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
+// 32-byte store: one full sector per lane (rows of the output are written by one thread each)
+__device__ __forceinline__ void st_global_v8(void* ptr, const uint32_t (&v)[8]) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(ptr), "r"(v[0]), "r"(v[1]), "r"(v[2]),
+               "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
+}
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&h);
@@ -304,7 +310,7 @@ struct TmaArgs {
 };
 
 __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_constant__ AttnParams p, int lg,
-                                                              int tile_major,
+                                                              int tile_major, int wide_store,
                                                               const __grid_constant__ TmaArgs tma) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -357,7 +363,26 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   const int32_t* kv_off = pl.kv_off + (size_t)map * (P + 1);
   const int32_t* vis = pl.vis + (size_t)map * pl.n_q * P;
   const int k_begin = p.fused ? 0 : part, k_end = p.fused ? P : part + 1;
-  if (warp == 0) {
+  // Query sub-tiles (row r = slot r / Gp, head r % Gp): the 128 softmax threads of a sub-tile gather it from the
+  // caller's tensor, 16 bytes per thread and row, half a warp per 256-byte row.  The loads are issued here, before the
+  // set-up below, and land in shared memory (128-byte-swizzled [2][128][128 B] layout) after it.  Rows past the end
+  // of the sub-tile repeat its last row (their results are discarded).
+  uint4 qv[16];
+  const int q_chunk = tid & 15;
+  if (warp < 8 && (warp >> 2) < n_sub) {
+    const int s = warp >> 2;
+    const int sub_row0 = row0 + s * R;
+    const int sub_nrows = min(R, nrows - s * R);
+    const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(p.q) + (int64_t)b * p.qs.batch + q_chunk * 8;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const int r = (tid >> 4 & 7) + 8 * j;
+      const int tok = __ldg(q_idx + sub_row0 + min(r >> lg, sub_nrows - 1));
+      qv[j] = __ldg(reinterpret_cast<const uint4*>(qb + (int64_t)tok * p.qs.token +
+                                                   (int64_t)(h0 + (r & (Gp - 1))) * p.qs.head));
+    }
+  }
+  if (warp == 11) {  // the warp without a role of its own
     // Compact the shards of which the CTA's last row (longest prefix; rows ascend) sees something, with what the
     // roles need per shard, and count the chunks of the stream.
     const int32_t* need_of = vis + (size_t)(row0 + nrows - 1) * P;
@@ -451,25 +476,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       float m_true = -INFINITY;  // exact running max
       float l_run = 0.f;
       if (n_tiles > 0) {
-        // Query sub-tile (row r = slot r / Gp, head r % Gp): this group's 128 threads gather it from the caller's tensor
-        // while they have nothing else to do, 16 bytes per thread and row, half a warp per 256-byte row, into the
-        // 128-byte-swizzled [2][128][128 B] layout.  Rows past the end of the sub-tile repeat its last row (their
-        // results are discarded).
-        const int chunk = m & 15;
-        const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(p.q) + (int64_t)b * p.qs.batch + chunk * 8;
-        uint4 qv[16];
+        uint8_t* q_tile = smem + kOffQ + s * kTileBytes + (q_chunk >> 3) * kHalfBytes;
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          const int r = (m >> 4) + 8 * j;
-          const int tok = __ldg(q_idx + sub_row0 + min(r >> lg, sub_nrows - 1));
-          qv[j] = __ldg(reinterpret_cast<const uint4*>(qb + (int64_t)tok * p.qs.token +
-                                                       (int64_t)(h0 + (r & (Gp - 1))) * p.qs.head));
-        }
-        uint8_t* q_tile = smem + kOffQ + s * kTileBytes + (chunk >> 3) * kHalfBytes;
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const int r = (m >> 4) + 8 * j;
-          *reinterpret_cast<uint4*>(q_tile + r * 128 + (((chunk & 7) ^ (r & 7)) << 4)) = qv[j];
+          const int r = (tid >> 4 & 7) + 8 * j;
+          *reinterpret_cast<uint4*>(q_tile + r * 128 + (((q_chunk & 7) ^ (r & 7)) << 4)) = qv[j];
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> tensor-core reads
         mbar_arrive(bar(Q_FULL + s));
@@ -633,13 +644,17 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
         }
         if (row_ok) {
 #pragma unroll
-          for (int j = 0; j < 32; j += 8) {
-            uint4 val;
-            val.x = pack_bf16x2(__uint_as_float(o[j]) * o_scale, __uint_as_float(o[j + 1]) * o_scale);
-            val.y = pack_bf16x2(__uint_as_float(o[j + 2]) * o_scale, __uint_as_float(o[j + 3]) * o_scale);
-            val.z = pack_bf16x2(__uint_as_float(o[j + 4]) * o_scale, __uint_as_float(o[j + 5]) * o_scale);
-            val.w = pack_bf16x2(__uint_as_float(o[j + 6]) * o_scale, __uint_as_float(o[j + 7]) * o_scale);
-            *reinterpret_cast<uint4*>(dst + cc * 32 + j) = val;
+          for (int j = 0; j < 32; j += 16) {
+            uint32_t val[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              val[e] = pack_bf16x2(__uint_as_float(o[j + 2 * e]) * o_scale, __uint_as_float(o[j + 2 * e + 1]) * o_scale);
+            if (wide_store) {
+              st_global_v8(dst + cc * 32 + j, val);
+            } else {
+              *reinterpret_cast<uint4*>(dst + cc * 32 + j) = make_uint4(val[0], val[1], val[2], val[3]);
+              *reinterpret_cast<uint4*>(dst + cc * 32 + j + 8) = make_uint4(val[4], val[5], val[6], val[7]);
+            }
           }
         }
       }
@@ -819,7 +834,12 @@ cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void
   const int64_t n_ctas = (int64_t)p.plan.n_qtiles[3 - lg] * (p.H >> lg) * p.batch * n_parts;
   if (n_ctas >= (int64_t)1 << 31) return cudaErrorInvalidConfiguration;
   const int tile_major = n_ctas <= 8 * 148;  // few CTAs per SM: balance matters more than L2 locality
-  tc::attn_tc_kernel<<<(unsigned)n_ctas, tc::kThreads, tc::kSmemBytes, stream>>>(p, lg, tile_major, tma);
+  // 32-byte stores of the output rows need 32-byte aligned rows (the interface only asks for 16)
+  const auto a32 = [](const void* ptr) { return ((uintptr_t)ptr & 31) == 0; };
+  const int wide_store = p.fused ? a32(p.o_out) && (p.os.batch * 2) % 32 == 0 && (p.os.token * 2) % 32 == 0 &&
+                                       (p.os.head * 2) % 32 == 0
+                                 : a32(p.o_part);
+  tc::attn_tc_kernel<<<(unsigned)n_ctas, tc::kThreads, tc::kSmemBytes, stream>>>(p, lg, tile_major, wide_store, tma);
   count_launch();
   return cudaGetLastError();
 }

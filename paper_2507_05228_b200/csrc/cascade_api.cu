@@ -426,8 +426,8 @@ static bool use_decode(const cascade_plan_t* plan, cascade_dtype_t dtype, int H,
   return plan->dev.n_q == 1 && dtype == CASCADE_BF16 && d == 128 && (G == 1 || G == 2 || G == 4 || G == 8);
 }
 static bool use_tc(const cascade_plan_t* plan, cascade_dtype_t dtype, int d) {
-  // the tensor-core kernel keeps per-shard bookkeeping in shared memory: at most 88 KV shards
-  return dtype == CASCADE_BF16 && d == 128 && plan->dev.n_q > 1 && plan->dev.n_kv_shards <= 88;
+  // the tensor-core kernel keeps per-shard bookkeeping in shared memory: at most 256 KV shards
+  return dtype == CASCADE_BF16 && d == 128 && plan->dev.n_q > 1 && plan->dev.n_kv_shards <= 256;
 }
 
 // Shard-major K and V copies for the tensor-core path: two regions of batch * kv_heads * n_kv rows of 256 bytes.
