@@ -82,6 +82,17 @@ const char* cascade_last_error(void);
 int64_t cascade_launch_count(void);
 
 /*
+ * Device-side timing of the attention kernel (for roofline accounting; not a step of the method).  Between
+ * cascade_kernel_timing_begin() and cascade_kernel_timing_end() every launch of the tensor-core attention kernel or of
+ * the decode kernel is bracketed by a pair of CUDA events recorded on the launch stream (at most 8192 launches; later
+ * ones are not timed).  cascade_kernel_timing_end SYNCHRONISES the device, stops the recording and returns the summed
+ * duration in milliseconds and the number of timed launches (either pointer may be NULL).  The shard-gather and merge
+ * launches are not included.  Not thread-safe against concurrent attention calls.  Errors: CUDA.
+ */
+cascade_status_t cascade_kernel_timing_begin(void);
+cascade_status_t cascade_kernel_timing_end(double* total_ms, int64_t* n_launches);
+
+/*
  * cascade_shard_plan -- index maps and causal pair mask (Section 5.1 index sets; Section 5.2.2 sorted
  * concatenation; the sharded mask s^{S_j T_k} = s[:, S_j, T_k]).
  * Because each shard is kept in ascending token order and the mask is unidirectional, row r of pair

@@ -28,6 +28,7 @@ EXPORTS = [
     "cascade_plan_destroy",
     "cascade_plan_get", "cascade_plan_dense_mask", "cascade_plan_device_status", "cascade_attn_partials",
     "cascade_merge", "cascade_attn_sharded", "cascade_workspace_bytes", "cascade_attn_decode_static",
+    "cascade_kernel_timing_begin", "cascade_kernel_timing_end",
 ]
 
 
@@ -71,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.cascade_attn_decode_static.argtypes = [vp, i32, i32, i32, f32, vp, Strides, vp, Strides, vp, Strides, vp,
                                                  Strides, vp, vp]
         L.cascade_workspace_bytes.argtypes = [vp, i32, i32, i32, i32, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
+        L.cascade_kernel_timing_begin.argtypes = []
+        L.cascade_kernel_timing_end.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
         for name in EXPORTS:
             if name not in ("cascade_version", "cascade_last_error", "cascade_launch_count"):
                 getattr(L, name).restype = i32
@@ -106,6 +109,17 @@ def cascade_version() -> int:
 
 def cascade_launch_count() -> int:
     return int(lib().cascade_launch_count())
+
+
+def cascade_kernel_timing_begin() -> None:
+    _check(lib().cascade_kernel_timing_begin())
+
+
+def cascade_kernel_timing_end():
+    """(summed milliseconds, launches) of the attention / decode kernels launched since ..._begin()."""
+    ms, n = ctypes.c_double(), ctypes.c_int64()
+    _check(lib().cascade_kernel_timing_end(ctypes.byref(ms), ctypes.byref(n)))
+    return ms.value, n.value
 
 
 class Plan:

@@ -839,6 +839,7 @@ cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void
   const int wide_store = p.fused ? a32(p.o_out) && (p.os.batch * 2) % 32 == 0 && (p.os.token * 2) % 32 == 0 &&
                                        (p.os.head * 2) % 32 == 0
                                  : a32(p.o_part);
+  TimedLaunch timed(stream);
   tc::attn_tc_kernel<<<(unsigned)n_ctas, tc::kThreads, tc::kSmemBytes, stream>>>(p, lg, tile_major, wide_store, tma);
   count_launch();
   return cudaGetLastError();

@@ -23,6 +23,30 @@ void set_error(const char* fmt, ...) {
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+// ---- kernel timing
+static bool g_timing_on = false;
+static std::vector<cudaEvent_t> g_ev_start, g_ev_stop;
+static size_t g_timed = 0;  // launches bracketed since begin
+constexpr size_t kMaxTimedLaunches = 8192;
+
+void timing_mark(cudaStream_t stream, bool start) {
+  if (!g_timing_on) return;
+  if (start) {
+    if (g_timed >= kMaxTimedLaunches) return;
+    if (g_ev_start.size() <= g_timed) {
+      cudaEvent_t a = nullptr, b = nullptr;
+      if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) return;
+      g_ev_start.push_back(a);
+      g_ev_stop.push_back(b);
+    }
+    cudaEventRecord(g_ev_start[g_timed], stream);
+  } else {
+    if (g_timed >= kMaxTimedLaunches || g_ev_start.size() <= g_timed) return;
+    cudaEventRecord(g_ev_stop[g_timed], stream);
+    ++g_timed;
+  }
+}
+
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 static cascade_status_t cuda_fail(cudaError_t e, const char* what) {
@@ -62,6 +86,28 @@ extern "C" {
 int32_t cascade_version(void) { return 100; }
 const char* cascade_last_error(void) { return g_err; }
 int64_t cascade_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+cascade_status_t cascade_kernel_timing_begin(void) {
+  g_timed = 0;
+  g_timing_on = true;
+  return CASCADE_OK;
+}
+
+cascade_status_t cascade_kernel_timing_end(double* total_ms, int64_t* n_launches) {
+  g_timing_on = false;
+  cudaError_t e = cudaDeviceSynchronize();
+  double sum = 0.0;
+  for (size_t i = 0; i < g_timed && e == cudaSuccess; ++i) {
+    float ms = 0.f;
+    e = cudaEventElapsedTime(&ms, g_ev_start[i], g_ev_stop[i]);
+    sum += ms;
+  }
+  if (total_ms) *total_ms = sum;
+  if (n_launches) *n_launches = (int64_t)g_timed;
+  g_timed = 0;
+  if (e != cudaSuccess) return cuda_fail(e, "cascade_kernel_timing_end");
+  return CASCADE_OK;
+}
 
 static cascade_status_t plan_host(int32_t n_maps, int32_t n_q, int32_t n_kv, const int32_t* q_shard_of,
                                   const int32_t* kv_shard_of, int32_t n_q_shards, int32_t n_kv_shards,

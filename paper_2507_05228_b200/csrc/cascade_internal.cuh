@@ -81,6 +81,13 @@ namespace cascade {
 
 void set_error(const char* fmt, ...);
 void count_launch(int n = 1);
+// Kernel timing (cascade_kernel_timing_begin / _end): brackets a launch with events when recording is on.
+void timing_mark(cudaStream_t stream, bool start);
+struct TimedLaunch {  // RAII: events around the launches issued while it lives
+  cudaStream_t st;
+  explicit TimedLaunch(cudaStream_t s) : st(s) { timing_mark(st, true); }
+  ~TimedLaunch() { timing_mark(st, false); }
+};
 
 // Launchers; each returns a cudaError_t from the launch.
 cudaError_t launch_attn_simt(const AttnParams& p, cascade_dtype_t dtype, cudaStream_t stream);

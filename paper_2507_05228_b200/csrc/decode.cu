@@ -201,6 +201,7 @@ __global__ void __launch_bounds__(128, 3) decode_kernel(AttnParams p) {
 
 cudaError_t launch_decode(const AttnParams& p, cudaStream_t stream) {
   dim3 grid(p.plan.n_kv_shards, p.Hkv, p.batch);
+  TimedLaunch timed(stream);
   switch (p.G) {
     case 1: decode_kernel<1><<<grid, 128, 0, stream>>>(p); break;
     case 2: decode_kernel<2><<<grid, 128, 0, stream>>>(p); break;
