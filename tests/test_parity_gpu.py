@@ -163,3 +163,54 @@ def test_workspace_contract_for_decode(gu):
     o_ref, lse_ref = oracle.attention_unsharded(w.q, w.k, w.v, w.scale, q_pos_offset=w.q_pos_offset)
     gu.check_output(o, None, o_ref, lse_ref, w.tol, "decode with caller workspace")
     plan.destroy()
+
+
+def test_many_small_shards_tiles_span_several_shards(gu):
+    """64 shards of 16 keys: every 32-key chunk of the KV stream is half empty and an MMA tile takes its four chunks
+    from four different shards; 300 shards exceed the tensor-core kernel's shard table and take the ALU kernel."""
+    gu.full_parity(wl.make_workload("shards64", 1, 1024, 1024, 8, 2, 128, "bf16", "random", "random", 64, 64, seed=11))
+    gu.full_parity(wl.make_workload("shards300", 1, 600, 600, 4, 2, 128, "bf16", "random", "random", 300, 300,
+                                    seed=12))
+
+
+def test_tensor_core_route_workspace_contract_and_unaligned_output(gu):
+    from paper_2507_05228_b200 import binding as cb
+    w = wl.make_workload("ws_tc", 2, 300, 300, 8, 2, 128, "bf16", "random", "random", 3, 3, seed=13)
+    q, k, v = gu.to_device(w)
+    plan = gu.make_plan(w)
+    need = cb.cascade_workspace_bytes(plan, cb.CALL_SHARDED, cb.BF16, 2, 8, 2, 128)
+    assert need == cb.cascade_workspace_bytes(plan, cb.CALL_PARTIALS, cb.BF16, 2, 8, 2, 128)
+    assert need >= 2 * 2 * 2 * 300 * 256  # shard-major K and V copies
+    small = torch.empty(need - 256, dtype=torch.uint8, device="cuda")
+    for call in (cb.cascade_attn_sharded, cb.cascade_attn_partials):
+        with pytest.raises(cb.CascadeError) as ei:
+            call(plan, q, k, v, w.scale, workspace=small)
+        assert ei.value.status == 4
+    # an output whose rows are 16- but not 32-byte aligned takes the narrow-store epilogue
+    flat = torch.zeros(q.numel() + 8, dtype=torch.bfloat16, device="cuda")
+    o_view = flat[8:].view(q.shape)
+    assert o_view.data_ptr() % 32 == 16
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    o, lse = cb.cascade_attn_sharded(plan, q, k, v, w.scale, out=o_view, workspace=ws)
+    o_ref, lse_ref = oracle.attention_unsharded(w.q, w.k, w.v, w.scale)
+    gu.check_output(o, lse, o_ref, lse_ref, w.tol, "unaligned output")
+    assert (flat[:8] == 0).all()
+    assert plan.device_status() == 0
+    plan.destroy()
+
+
+def test_kernel_timing_counts_attention_launches(gu):
+    from paper_2507_05228_b200 import binding as cb
+    w = wl.make_workload("timing", 1, 256, 256, 8, 2, 128, "bf16", "random", "random", 2, 2, seed=14)
+    q, k, v = gu.to_device(w)
+    plan = gu.make_plan(w)
+    cb.cascade_attn_sharded(plan, q, k, v, w.scale)  # not timed
+    cb.cascade_kernel_timing_begin()
+    for _ in range(3):
+        cb.cascade_attn_sharded(plan, q, k, v, w.scale)
+    ms, n = cb.cascade_kernel_timing_end()
+    assert n == 3 and 0.0 < ms < 100.0
+    cb.cascade_attn_sharded(plan, q, k, v, w.scale)  # recording is off again
+    ms2, n2 = cb.cascade_kernel_timing_end()
+    assert n2 == 0 and ms2 == 0.0
+    plan.destroy()
