@@ -211,6 +211,9 @@ def run_ours(args):
                 "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"], "frac_of_nominal_2250": achieved / 2250.0,
                 "kernel_ms": kernel_ms, "kernel_launches_timed": kernel_launches,
                 "traffic": NCU_TRAFFIC_BYTES.get(HEADLINE)}
+    if rank == 0 and world == 1 and not args.no_extras:
+        routes["fused_rope"] = _rope_record(torch, cb, w, plan, q, k, v, o, ws, flush, routes["fused"]["ms"], kernel_ms,
+                                            steps=max(args.steps, 20))
     plan.destroy()
     del q, k, v, o, parts
 
@@ -245,6 +248,24 @@ def run_ours(args):
     cd.finalize()
 
 
+ROPE_BASE = 500000.0  # rotary base of the model family the prefill shapes are taken from
+
+
+def _rope_record(torch, cb, w, plan, q, k, v, o, ws, flush, plain_ms, plain_kernel_ms, steps=5):
+    """The fused route with the rotary step of the pre-pass folded into the staging of Q and K rows: what the extra
+    arithmetic costs over the same call on rotated inputs (a separate rotary pass would read and write Q and K once)."""
+    table = cb.cascade_rope_table(max(w.q_pos_offset + w.n_q, w.n_kv), w.d, ROPE_BASE)
+    ms = _time_steps(torch, lambda: cb.cascade_attn_sharded_rope(plan, q, k, v, w.scale, table, out=o, want_lse=False,
+                                                                 workspace=ws), steps, 3, flush,
+                     after_warmup=cb.cascade_kernel_timing_begin)
+    k_ms, k_n = cb.cascade_kernel_timing_end()
+    med = statistics.median(ms)
+    qk_bytes = 2 * (w.B * w.n_q * w.H + w.B * w.n_kv * w.Hkv) * w.d * 2  # one read + one write of Q and K
+    return {"rope_fused_ms": med, "rope_attn_kernel_ms": k_ms / max(k_n, 1), "rope_extra_ms": med - plain_ms,
+            "rope_attn_kernel_extra_ms": k_ms / max(k_n, 1) - plain_kernel_ms,
+            "separate_rotary_pass_bytes": qk_bytes}
+
+
 def run_extras(torch, cb, wl, flush, peaks):
     """The other prefill workloads (tensor-bound) and the decode step and merge (HBM-bound), a few steps each."""
     out = {}
@@ -265,6 +286,7 @@ def run_extras(torch, cb, wl, flush, peaks):
                "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"], "frac_of_nominal_2250": tf / 2250.0,
                "attn_kernel_ms": k_ms / max(k_n, 1), "attn_kernel_tflops": ktf,
                "attn_kernel_frac_of_burst_peak": ktf / peaks["bf16_tflops"]}
+        rec.update(_rope_record(torch, cb, w, plan, q, k, v, o, ws, flush, rec["fused_ms"], rec["attn_kernel_ms"]))
         # unfused route: partials (tensor) then merge (HBM)
         parts = cb.cascade_attn_partials(plan, q, k, v, w.scale, workspace=ws)
         ms_p = _time_steps(torch, lambda: cb.cascade_attn_partials(plan, q, k, v, w.scale, out=parts, workspace=ws), 3, 2,

@@ -195,6 +195,43 @@ cascade_status_t cascade_attn_sharded(const cascade_plan_t* plan, cascade_dtype_
                                       size_t workspace_bytes, void* stream);
 
 /*
+ * cascade_rope_table -- the positional table p of the rotary embedding (Section 4 lists p among the tensors set up
+ * before inference and sharded with the tokens; Algorithm 2 consumes its rows p^{R_i}).  The paper does not print
+ * the rotary formula; this library takes the rotate-half form with theta_i = base^(-2 i / head_dim):
+ *   table[t][i] = (cos(t theta_i), sin(t theta_i)),  t = 0 .. n_positions-1,  i = 0 .. head_dim/2 - 1,
+ * angles formed and evaluated in fp64, stored as fp32 pairs.
+ *   table  DEVICE fp32 [n_positions][head_dim/2][2], 16-byte aligned, caller-owned; written on `stream`.
+ * Errors: CASCADE_ERR_INVALID_ARG (null / misaligned table, n_positions < 1, odd head_dim, base <= 1),
+ * CASCADE_ERR_CUDA (launch failure).
+ */
+cascade_status_t cascade_rope_table(int32_t n_positions, int32_t head_dim, double base, float* table,
+                                    void* stream);
+
+/*
+ * cascade_attn_sharded_rope -- cascade_attn_sharded with the tail of the pre-pass fused in (Algorithm 2:
+ * q <- rotary_pos_emb(q, p^{R_i}), k <- rotary_pos_emb(k, p^{R_i})): q and k are given UNROTATED; every query row is
+ * turned by the table row of its position (q_pos_offset + token index) and every key row by the row of its token
+ * index while they are staged for the attention kernel, so no separate pass over q and k runs:
+ *   y[i] = x[i] cos - x[i + d/2] sin,   y[i + d/2] = x[i + d/2] cos + x[i] sin,   (cos, sin) = table[pos][i],
+ * computed in fp32 and rounded once to bf16, the type the pre-pass would hand q and k on in.  Because a row's angle
+ * depends on its original index only, the result equals rotating the whole sequence first and calling
+ * cascade_attn_sharded.
+ *   rope_table   DEVICE table written by cascade_rope_table for head_dim 128, 16-byte aligned, read-only
+ *   n_positions  its row count; must cover max(q_pos_offset + n_q, n_kv)
+ * All other arguments, the workspace and the outputs are those of cascade_attn_sharded.
+ * Supported on the tensor-core route only (bf16, head_dim 128, n_q > 1, at most 256 KV shards); other shapes return
+ * CASCADE_ERR_UNSUPPORTED and the caller rotates q and k beforehand.
+ */
+cascade_status_t cascade_attn_sharded_rope(const cascade_plan_t* plan, cascade_dtype_t dtype, int32_t batch,
+                                           int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, float scale,
+                                           const void* q, cascade_strides_t q_strides, const void* k,
+                                           cascade_strides_t k_strides, const void* v,
+                                           cascade_strides_t v_strides, const float* rope_table,
+                                           int32_t n_positions, void* o_out, cascade_strides_t o_strides,
+                                           float* lse_out, void* workspace, size_t workspace_bytes,
+                                           void* stream);
+
+/*
  * cascade_attn_decode_static -- the decode case of cascade_attn_sharded (one query row per sequence, bf16,
  * head_dim 128, n_heads / n_kv_heads in {1,2,4,8}) without a workspace argument and without any allocation.
  * (The paper has no counterpart: this is a convenience of this library, not a step of the method.)

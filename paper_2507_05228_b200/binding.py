@@ -28,7 +28,7 @@ EXPORTS = [
     "cascade_plan_destroy",
     "cascade_plan_get", "cascade_plan_dense_mask", "cascade_plan_device_status", "cascade_attn_partials",
     "cascade_merge", "cascade_attn_sharded", "cascade_workspace_bytes", "cascade_attn_decode_static",
-    "cascade_kernel_timing_begin", "cascade_kernel_timing_end",
+    "cascade_kernel_timing_begin", "cascade_kernel_timing_end", "cascade_rope_table", "cascade_attn_sharded_rope",
 ]
 
 
@@ -72,6 +72,9 @@ def lib() -> ctypes.CDLL:
         L.cascade_attn_decode_static.argtypes = [vp, i32, i32, i32, f32, vp, Strides, vp, Strides, vp, Strides, vp,
                                                  Strides, vp, vp]
         L.cascade_workspace_bytes.argtypes = [vp, i32, i32, i32, i32, i32, i32, ctypes.POINTER(ctypes.c_size_t)]
+        L.cascade_rope_table.argtypes = [i32, i32, ctypes.c_double, vp, vp]
+        L.cascade_attn_sharded_rope.argtypes = [vp, i32, i32, i32, i32, i32, f32, vp, Strides, vp, Strides, vp, Strides,
+                                                vp, i32, vp, Strides, vp, vp, ctypes.c_size_t, vp]
         L.cascade_kernel_timing_begin.argtypes = []
         L.cascade_kernel_timing_end.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
         for name in EXPORTS:
@@ -275,6 +278,31 @@ def cascade_attn_sharded(plan: Plan, q: torch.Tensor, k: torch.Tensor, v: torch.
                                       k.data_ptr(), _strides(k), v.data_ptr(), _strides(v), o.data_ptr(),
                                       _strides(o), lse.data_ptr() if lse is not None else None, ws_ptr, ws_bytes,
                                       _stream()))
+    return o, lse
+
+
+def cascade_rope_table(n_positions: int, head_dim: int, base: float, device="cuda") -> torch.Tensor:
+    """Positional table of the rotary embedding on the device: fp32 [n_positions, head_dim/2, 2] = (cos, sin)."""
+    table = torch.empty((n_positions, head_dim // 2, 2), dtype=torch.float32, device=device)
+    _check(lib().cascade_rope_table(n_positions, head_dim, float(base), table.data_ptr(), _stream()))
+    return table
+
+
+def cascade_attn_sharded_rope(plan: Plan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, scale: float,
+                              rope_table: torch.Tensor, out=None, want_lse: bool = True, workspace=None):
+    """cascade_attn_sharded on unrotated q, k with the rotary step fused into the staging of their rows."""
+    B, n_q, H, d = q.shape
+    Hkv = k.shape[2]
+    code = _dtype_code(q)
+    assert rope_table.dtype == torch.float32 and rope_table.is_contiguous() and rope_table.shape[1:] == (d // 2, 2)
+    o = out if out is not None else torch.empty((B, n_q, H, d), dtype=q.dtype, device=q.device)
+    lse = torch.empty((B, n_q, H), dtype=torch.float32, device=q.device) if want_lse else None
+    nbytes = cascade_workspace_bytes(plan, CALL_SHARDED, code, B, H, Hkv, d)
+    ws, ws_ptr, ws_bytes = _ws(nbytes, q.device, workspace)
+    _check(lib().cascade_attn_sharded_rope(plan.handle, code, B, H, Hkv, d, scale, q.data_ptr(), _strides(q),
+                                           k.data_ptr(), _strides(k), v.data_ptr(), _strides(v),
+                                           rope_table.data_ptr(), rope_table.shape[0], o.data_ptr(), _strides(o),
+                                           lse.data_ptr() if lse is not None else None, ws_ptr, ws_bytes, _stream()))
     return o, lse
 
 

@@ -309,6 +309,9 @@ struct TmaArgs {
   CUtensorMap k, v;  // shard-major copies as [batch * kv_heads][n_kv][head_dim]
 };
 
+// kRope: the query rows are turned by the rotary embedding of their positions while they are staged (the key rows
+// were turned by the gather pass), Algorithm 2.
+template <bool kRope>
 __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_constant__ AttnParams p, int lg,
                                                               int tile_major, int wide_store,
                                                               const __grid_constant__ TmaArgs tma) {
@@ -369,17 +372,39 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   // of the sub-tile repeat its last row (their results are discarded).
   uint4 qv[16];
   const int q_chunk = tid & 15;
+  const float4* rope_row[kRope ? 8 : 1];  // this thread's slice of the table row of each of its query rows
+  float4 cs[kRope ? 4 : 1][4];            // (cos, sin) of four rows: 8 pairs each
   if (warp < 8 && (warp >> 2) < n_sub) {
     const int s = warp >> 2;
     const int sub_row0 = row0 + s * R;
     const int sub_nrows = min(R, nrows - s * R);
-    const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(p.q) + (int64_t)b * p.qs.batch + q_chunk * 8;
+    if constexpr (kRope) {
+      // Rotary staging: a thread holds both halves of 8 rotation pairs of a row (columns 8 c .. and 64 + 8 c ..),
+      // 8 threads per row, 8 rows per thread, and the (cos, sin) of the first four of its rows; the table rows of the
+      // other four are fetched while those are turned.
+      const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(p.q) + (int64_t)b * p.qs.batch + (tid & 7) * 8;
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      const int r = (tid >> 4 & 7) + 8 * j;
-      const int tok = __ldg(q_idx + sub_row0 + min(r >> lg, sub_nrows - 1));
-      qv[j] = __ldg(reinterpret_cast<const uint4*>(qb + (int64_t)tok * p.qs.token +
-                                                   (int64_t)(h0 + (r & (Gp - 1))) * p.qs.head));
+      for (int j = 0; j < 8; ++j) {
+        const int r = (tid >> 3 & 15) + 16 * j;
+        const int tok = __ldg(q_idx + sub_row0 + min(r >> lg, sub_nrows - 1));
+        const __nv_bfloat16* row = qb + (int64_t)tok * p.qs.token + (int64_t)(h0 + (r & (Gp - 1))) * p.qs.head;
+        qv[2 * j] = __ldg(reinterpret_cast<const uint4*>(row));
+        qv[2 * j + 1] = __ldg(reinterpret_cast<const uint4*>(row + 64));
+        rope_row[j] = reinterpret_cast<const float4*>(p.rope + (int64_t)(pl.q_pos_offset + tok) * 64 + (tid & 7) * 8);
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) cs[j][e] = __ldg(rope_row[j] + e);
+    } else {
+      const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(p.q) + (int64_t)b * p.qs.batch + q_chunk * 8;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const int r = (tid >> 4 & 7) + 8 * j;
+        const int tok = __ldg(q_idx + sub_row0 + min(r >> lg, sub_nrows - 1));
+        qv[j] = __ldg(reinterpret_cast<const uint4*>(qb + (int64_t)tok * p.qs.token +
+                                                     (int64_t)(h0 + (r & (Gp - 1))) * p.qs.head));
+      }
     }
   }
   if (warp == 11) {  // the warp without a role of its own
@@ -476,11 +501,41 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       float m_true = -INFINITY;  // exact running max
       float l_run = 0.f;
       if (n_tiles > 0) {
-        uint8_t* q_tile = smem + kOffQ + s * kTileBytes + (q_chunk >> 3) * kHalfBytes;
+if constexpr (kRope) {
+          // q <- rotary_pos_emb(q, p): (lo, hi) = (x[i], x[i + 64]) -> (lo cos - hi sin, hi cos + lo sin) in fp32,
+          // rounded once to bf16, then stored like the unrotated rows
+          uint8_t* q_tile = smem + kOffQ + s * kTileBytes;
+          const int c = tid & 7;
+          auto turn_and_store = [&](int j, const float4 (&t)[4]) {
+            __nv_bfloat162* lo = reinterpret_cast<__nv_bfloat162*>(&qv[2 * j]);
+            __nv_bfloat162* hi = reinterpret_cast<__nv_bfloat162*>(&qv[2 * j + 1]);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const int r = (tid >> 4 & 7) + 8 * j;
-          *reinterpret_cast<uint4*>(q_tile + r * 128 + (((q_chunk & 7) ^ (r & 7)) << 4)) = qv[j];
+            for (int e = 0; e < 4; ++e) {
+              const float2 a = __bfloat1622float2(lo[e]), h = __bfloat1622float2(hi[e]);
+              lo[e] = __floats2bfloat162_rn(a.x * t[e].x - h.x * t[e].y, a.y * t[e].z - h.y * t[e].w);
+              hi[e] = __floats2bfloat162_rn(h.x * t[e].x + a.x * t[e].y, h.y * t[e].z + a.y * t[e].w);
+            }
+            const int r = (tid >> 3 & 15) + 16 * j;
+            uint8_t* dst = q_tile + r * 128 + ((c ^ (r & 7)) << 4);
+            *reinterpret_cast<uint4*>(dst) = qv[2 * j];
+            *reinterpret_cast<uint4*>(dst + kHalfBytes) = qv[2 * j + 1];
+          };
+          float4 cs2[4][4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) cs2[j][e] = __ldg(rope_row[4 + j] + e);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) turn_and_store(j, cs[j]);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) turn_and_store(4 + j, cs2[j]);
+        } else {
+          uint8_t* q_tile = smem + kOffQ + s * kTileBytes + (q_chunk >> 3) * kHalfBytes;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int r = (tid >> 4 & 7) + 8 * j;
+            *reinterpret_cast<uint4*>(q_tile + r * 128 + (((q_chunk & 7) ^ (r & 7)) << 4)) = qv[j];
+          }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> tensor-core reads
         mbar_arrive(bar(Q_FULL + s));
@@ -818,8 +873,8 @@ bool encode_sorted(CUtensorMap* map, const void* base, int64_t n_kv, int64_t n_m
 }  // namespace
 
 cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void* v_sorted, cudaStream_t stream) {
-  cudaError_t e = cudaFuncSetAttribute(tc::attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       tc::kSmemBytes);
+  auto kernel = p.rope ? tc::attn_tc_kernel<true> : tc::attn_tc_kernel<false>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes);
   if (e != cudaSuccess) return e;
   tc::TmaArgs tma;
   const int64_t n_mats = (int64_t)p.batch * p.Hkv;
@@ -840,7 +895,7 @@ cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void
                                        (p.os.head * 2) % 32 == 0
                                  : a32(p.o_part);
   TimedLaunch timed(stream);
-  tc::attn_tc_kernel<<<(unsigned)n_ctas, tc::kThreads, tc::kSmemBytes, stream>>>(p, lg, tile_major, wide_store, tma);
+  kernel<<<(unsigned)n_ctas, tc::kThreads, tc::kSmemBytes, stream>>>(p, lg, tile_major, wide_store, tma);
   count_launch();
   return cudaGetLastError();
 }

@@ -609,32 +609,52 @@ cascade_status_t cascade_merge(cascade_dtype_t dtype, int32_t batch, int32_t n_p
   return CASCADE_OK;
 }
 
-cascade_status_t cascade_attn_sharded(const cascade_plan_t* plan, cascade_dtype_t dtype, int32_t batch,
-                                      int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, float scale,
-                                      const void* q, cascade_strides_t q_strides, const void* k,
-                                      cascade_strides_t k_strides, const void* v, cascade_strides_t v_strides,
-                                      void* o_out, cascade_strides_t o_strides, float* lse_out, void* workspace,
-                                      size_t workspace_bytes, void* stream) {
-  cascade_status_t s = check_attn_args("cascade_attn_sharded", plan, dtype, batch, n_heads, n_kv_heads,
-                                       head_dim, q, q_strides, k, k_strides, v, v_strides);
+}  // extern "C"
+
+// The fused route; rope_table != null adds the rotary step (cascade_attn_sharded_rope).
+static cascade_status_t attn_sharded_impl(const char* fn, const cascade_plan_t* plan, cascade_dtype_t dtype,
+                                          int32_t batch, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim,
+                                          float scale, const void* q, cascade_strides_t q_strides, const void* k,
+                                          cascade_strides_t k_strides, const void* v, cascade_strides_t v_strides,
+                                          const float* rope_table, int32_t n_positions, void* o_out,
+                                          cascade_strides_t o_strides, float* lse_out, void* workspace,
+                                          size_t workspace_bytes, void* stream) {
+  cascade_status_t s = check_attn_args(fn, plan, dtype, batch, n_heads, n_kv_heads, head_dim, q, q_strides, k,
+                                       k_strides, v, v_strides);
   if (s != CASCADE_OK) return s;
   if (!o_out) {
-    set_error("cascade_attn_sharded: null output pointer");
+    set_error("%s: null output pointer", fn);
     return CASCADE_ERR_INVALID_ARG;
   }
   if (!aligned16(o_out) || !strides_ok(o_strides, elt_size(dtype))) {
-    set_error("cascade_attn_sharded: output pointer and row strides must be 16-byte aligned");
+    set_error("%s: output pointer and row strides must be 16-byte aligned", fn);
     return CASCADE_ERR_INVALID_ARG;
   }
   AttnParams p = make_params(plan, batch, n_heads, n_kv_heads, head_dim, scale, q, q_strides, k, k_strides, v,
                              v_strides);
+  if (rope_table) {
+    if (!aligned16(rope_table)) {
+      set_error("%s: the positional table must be 16-byte aligned", fn);
+      return CASCADE_ERR_INVALID_ARG;
+    }
+    const int64_t need = std::max<int64_t>((int64_t)plan->dev.q_pos_offset + plan->dev.n_q, plan->dev.n_kv);
+    if (n_positions < need) {
+      set_error("%s: the positional table has %d rows, the plan needs %lld", fn, n_positions, (long long)need);
+      return CASCADE_ERR_INVALID_ARG;
+    }
+    if (use_decode(plan, dtype, n_heads, n_kv_heads, head_dim) || !use_tc(plan, dtype, head_dim)) {
+      set_error("%s: the rotary step is fused on the tensor-core route only (bf16, head_dim 128, more than one query "
+                "row, at most %d KV shards)", fn, 256);
+      return CASCADE_ERR_UNSUPPORTED;
+    }
+    p.rope = reinterpret_cast<const float2*>(rope_table);
+  }
   cudaStream_t st = (cudaStream_t)stream;
   if (use_decode(plan, dtype, n_heads, n_kv_heads, head_dim)) {
     // one query row per sequence: every KV shard is an independent partial, combined by the merge kernel
     const size_t need = decode_ws_bytes(plan, dtype, batch, n_heads, head_dim);
     if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255)) {
-      set_error("cascade_attn_sharded: workspace of %zu bytes (256-byte aligned) required, got %zu", need,
-                workspace_bytes);
+      set_error("%s: workspace of %zu bytes (256-byte aligned) required, got %zu", fn, need, workspace_bytes);
       return CASCADE_ERR_WORKSPACE;
     }
     const size_t rows = (size_t)batch * plan->dev.n_kv_shards * plan->dev.n_q * n_heads;
@@ -644,7 +664,7 @@ cascade_status_t cascade_attn_sharded(const cascade_plan_t* plan, cascade_dtype_
     p.m_part = (float*)(ws + align_up(rows * head_dim * elt_size(dtype), 256));
     p.l_part = (float*)((char*)p.m_part + align_up(rows * 4, 256));
     cudaError_t e = launch_decode(p, st);
-    if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_sharded: decode launch");
+    if (e != cudaSuccess) return cuda_fail(e, "attention (fused route): decode launch");
     MergeParams mp;
     mp.o_part = p.o_part;
     mp.m_part = p.m_part;
@@ -660,7 +680,7 @@ cascade_status_t cascade_attn_sharded(const cascade_plan_t* plan, cascade_dtype_
     mp.H = n_heads;
     mp.d = head_dim;
     e = launch_merge(mp, dtype, st);
-    if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_sharded: merge launch");
+    if (e != cudaSuccess) return cuda_fail(e, "attention (fused route): merge launch");
     return CASCADE_OK;
   }
   p.fused = 1;
@@ -669,12 +689,56 @@ cascade_status_t cascade_attn_sharded(const cascade_plan_t* plan, cascade_dtype_
   p.lse_out = lse_out;
   cudaError_t e;
   if (use_tc(plan, dtype, head_dim)) {
-    cascade_status_t ws = run_tc(p, "cascade_attn_sharded", plan, workspace, workspace_bytes, st, &e);
+    cascade_status_t ws = run_tc(p, fn, plan, workspace, workspace_bytes, st, &e);
     if (ws != CASCADE_OK) return ws;
   } else {
     e = launch_attn_simt(p, dtype, st);
   }
-  if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_sharded: launch");
+  if (e != cudaSuccess) return cuda_fail(e, "attention (fused route): launch");
+  return CASCADE_OK;
+}
+
+extern "C" {
+
+cascade_status_t cascade_attn_sharded(const cascade_plan_t* plan, cascade_dtype_t dtype, int32_t batch,
+                                      int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, float scale,
+                                      const void* q, cascade_strides_t q_strides, const void* k,
+                                      cascade_strides_t k_strides, const void* v, cascade_strides_t v_strides,
+                                      void* o_out, cascade_strides_t o_strides, float* lse_out, void* workspace,
+                                      size_t workspace_bytes, void* stream) {
+  return attn_sharded_impl("cascade_attn_sharded", plan, dtype, batch, n_heads, n_kv_heads, head_dim, scale, q,
+                           q_strides, k, k_strides, v, v_strides, nullptr, 0, o_out, o_strides, lse_out, workspace,
+                           workspace_bytes, stream);
+}
+
+cascade_status_t cascade_attn_sharded_rope(const cascade_plan_t* plan, cascade_dtype_t dtype, int32_t batch,
+                                           int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, float scale,
+                                           const void* q, cascade_strides_t q_strides, const void* k,
+                                           cascade_strides_t k_strides, const void* v, cascade_strides_t v_strides,
+                                           const float* rope_table, int32_t n_positions, void* o_out,
+                                           cascade_strides_t o_strides, float* lse_out, void* workspace,
+                                           size_t workspace_bytes, void* stream) {
+  if (!rope_table) {
+    set_error("cascade_attn_sharded_rope: null positional table");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  return attn_sharded_impl("cascade_attn_sharded_rope", plan, dtype, batch, n_heads, n_kv_heads, head_dim, scale, q,
+                           q_strides, k, k_strides, v, v_strides, rope_table, n_positions, o_out, o_strides, lse_out,
+                           workspace, workspace_bytes, stream);
+}
+
+cascade_status_t cascade_rope_table(int32_t n_positions, int32_t head_dim, double base, float* table, void* stream) {
+  if (!table || n_positions < 1 || head_dim < 2 || head_dim % 2 != 0 || !(base > 1.0)) {
+    set_error("cascade_rope_table: need a table pointer, n_positions >= 1, an even head_dim >= 2 and base > 1");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (!aligned16(table)) {
+    set_error("cascade_rope_table: the table must be 16-byte aligned");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  cudaError_t e = launch_rope_table(n_positions, head_dim, base, reinterpret_cast<float2*>(table),
+                                    (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e, "cascade_rope_table: launch");
   return CASCADE_OK;
 }
 

@@ -52,6 +52,10 @@ struct AttnParams {
   void* o_out;
   Strides os;
   float* lse_out;
+  // Rotary step of the pre-pass fused into the staging of Q and K rows (Algorithm 2): rows of the positional table,
+  // rope[position * 64 + i] = (cos, sin) of position * theta_i; null = rows are used as given.  A query row sits at
+  // position q_pos_offset + token, a key row at its token index.
+  const float2* rope;
 };
 
 struct MergeParams {
@@ -94,6 +98,7 @@ cudaError_t launch_attn_simt(const AttnParams& p, cascade_dtype_t dtype, cudaStr
 // k_sorted / v_sorted: the shard-major copies written by launch_gather_kv, [batch][kv_head][n_kv][128] bf16
 cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void* v_sorted, cudaStream_t stream);
 cudaError_t launch_gather_kv(const AttnParams& p, void* k_out, void* v_out, cudaStream_t stream);
+cudaError_t launch_rope_table(int32_t n_positions, int32_t head_dim, double base, float2* table, cudaStream_t stream);
 cudaError_t launch_decode(const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_merge(const MergeParams& p, cascade_dtype_t dtype, cudaStream_t stream);
 

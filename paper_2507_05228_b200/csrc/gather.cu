@@ -42,9 +42,98 @@ __global__ void __launch_bounds__(256) gather_kv_kernel(AttnParams p, __nv_bfloa
   }
 }
 
+// Turns the 8 pairs (lo[e], hi[e]) by the angles whose (cos, sin) are cs[0..7]: lo' = lo cos - hi sin,
+// hi' = hi cos + lo sin, in fp32, rounded once to bf16.
+__device__ __forceinline__ void rotate8(uint4& lo, uint4& hi, const float2* __restrict__ cs) {
+  const float4* cs4 = reinterpret_cast<const float4*>(cs);
+  __nv_bfloat162* l2 = reinterpret_cast<__nv_bfloat162*>(&lo);
+  __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&hi);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float4 t = __ldg(cs4 + e);  // (cos, sin) of pairs 2e and 2e + 1
+    const float2 a = __bfloat1622float2(l2[e]), b = __bfloat1622float2(h2[e]);
+    l2[e] = __floats2bfloat162_rn(a.x * t.x - b.x * t.y, a.y * t.z - b.y * t.w);
+    h2[e] = __floats2bfloat162_rn(b.x * t.x + a.x * t.y, b.y * t.z + a.y * t.w);
+  }
+}
+
+// The same gather with the rotary step of the pre-pass (Algorithm 2: k <- rotary_pos_emb(k, p^{R_i})) applied to the
+// key rows on the way: a key row is turned by the angles of its own token index, so the rotation needs nothing but
+// the row and its row of the positional table.  A thread holds both halves of 8 rotation pairs (columns 8c.. and
+// 64 + 8c..), 8 threads per row; V rows are copied as they are.
+__global__ void __launch_bounds__(256) gather_kv_rope_kernel(AttnParams p, __nv_bfloat16* k_out, __nv_bfloat16* v_out) {
+  constexpr int D = 128;
+  constexpr int kPasses = kGatherRowsPerCta / 32;
+  const PlanDev& pl = p.plan;
+  const int g = blockIdx.y, b = blockIdx.z;
+  const int map = pl.n_maps == 1 ? 0 : b;
+  const int32_t* kv_idx = pl.kv_idx + (size_t)map * pl.n_kv;
+  const int chunk = threadIdx.x & 7, r0 = threadIdx.x >> 3;  // 32 rows per pass
+  const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(p.k) + (int64_t)b * p.ks.batch + (int64_t)g * p.ks.head;
+  const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(p.v) + (int64_t)b * p.vs.batch + (int64_t)g * p.vs.head;
+  const int64_t out_base = ((int64_t)b * p.Hkv + g) * pl.n_kv;
+  const int slot0 = blockIdx.x * kGatherRowsPerCta;
+  uint4 klo[kPasses], khi[kPasses], vlo[kPasses], vhi[kPasses];
+  int tok[kPasses];
+#pragma unroll
+  for (int i = 0; i < kPasses; ++i) {
+    const int slot = slot0 + 32 * i + r0;
+    if (slot < pl.n_kv) {
+      tok[i] = __ldg(kv_idx + slot);
+      const __nv_bfloat16* kr = kb + (int64_t)tok[i] * p.ks.token + chunk * 8;
+      const __nv_bfloat16* vr = vb + (int64_t)tok[i] * p.vs.token + chunk * 8;
+      klo[i] = __ldcs(reinterpret_cast<const uint4*>(kr));
+      khi[i] = __ldcs(reinterpret_cast<const uint4*>(kr + 64));
+      vlo[i] = __ldcs(reinterpret_cast<const uint4*>(vr));
+      vhi[i] = __ldcs(reinterpret_cast<const uint4*>(vr + 64));
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kPasses; ++i) {
+    const int slot = slot0 + 32 * i + r0;
+    if (slot < pl.n_kv) {
+      rotate8(klo[i], khi[i], p.rope + (int64_t)tok[i] * (D / 2) + chunk * 8);
+      __nv_bfloat16* ko = k_out + (out_base + slot) * D + chunk * 8;
+      __nv_bfloat16* vo = v_out + (out_base + slot) * D + chunk * 8;
+      *reinterpret_cast<uint4*>(ko) = klo[i];
+      *reinterpret_cast<uint4*>(ko + 64) = khi[i];
+      *reinterpret_cast<uint4*>(vo) = vlo[i];
+      *reinterpret_cast<uint4*>(vo + 64) = vhi[i];
+    }
+  }
+}
+
 cudaError_t launch_gather_kv(const AttnParams& p, void* k_out, void* v_out, cudaStream_t stream) {
   dim3 grid((p.plan.n_kv + kGatherRowsPerCta - 1) / kGatherRowsPerCta, p.Hkv, p.batch);
-  gather_kv_kernel<<<grid, 256, 0, stream>>>(p, static_cast<__nv_bfloat16*>(k_out), static_cast<__nv_bfloat16*>(v_out));
+  if (p.rope) {
+    gather_kv_rope_kernel<<<grid, 256, 0, stream>>>(p, static_cast<__nv_bfloat16*>(k_out),
+                                                    static_cast<__nv_bfloat16*>(v_out));
+  } else {
+    gather_kv_kernel<<<grid, 256, 0, stream>>>(p, static_cast<__nv_bfloat16*>(k_out),
+                                               static_cast<__nv_bfloat16*>(v_out));
+  }
+  count_launch();
+  return cudaGetLastError();
+}
+
+// Positional table p of the rotary embedding (Section 4: p is set up before inference; Algorithm 2 takes its rows
+// p^{R_i}): table[t * d/2 + i] = (cos, sin)(t * base^(-2 i / d)), angles formed and evaluated in fp64, stored as fp32.
+__global__ void __launch_bounds__(256) rope_table_kernel(int32_t n_positions, int32_t half, double base,
+                                                         float2* __restrict__ table) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)n_positions * half) return;
+  const int i = (int)(idx % half);
+  const double t = (double)(idx / half);
+  const double theta = pow(base, -(double)i / (double)half);
+  double s, c;
+  sincos(t * theta, &s, &c);
+  table[idx] = make_float2((float)c, (float)s);
+}
+
+cudaError_t launch_rope_table(int32_t n_positions, int32_t head_dim, double base, float2* table, cudaStream_t stream) {
+  const int half = head_dim / 2;
+  const int64_t n = (int64_t)n_positions * half;
+  rope_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(n_positions, half, base, table);
   count_launch();
   return cudaGetLastError();
 }
