@@ -126,3 +126,59 @@ def test_visible_pair_count_matches_closed_form():
     plan = oracle.shard_plan(w.q_shard_of, w.kv_shard_of, w.n_q_shards, w.n_kv_shards)
     assert int(plan.vis.sum()) == 256 * 257 // 2 == w.visible_pairs()
     assert w.flops() == 4 * 128 * 4 * (256 * 257 // 2)
+
+
+def test_gaps_of_the_paper_example_and_closed_forms():
+    """Section 6.2: in a (c, delta)-sequence the distance from one cluster to the next is delta - c + 1, i.e. delta - c
+    indices lie between them; Section 6.3: (c, delta)-sharding meets the theorem iff delta - c + 1 >= rho + 1."""
+    g = _golden()
+    # R_1 = {1,2,7,8,13,14}: three clusters, four unknown tokens between neighbours (delta - c = 4)
+    assert sharding.index_set_gaps(g["R_1"]) == {"n_indices": 6, "n_clusters": 3, "min_gap": 4, "max_gap": 4}
+    # AttnNode set S_1121 = {1,3,7,9,13,15}: six singletons, gaps 1,3,1,3,1
+    assert sharding.index_set_gaps(g["S_1121"]) == {"n_indices": 6, "n_clusters": 6, "min_gap": 1, "max_gap": 3}
+    # S_1112 = R_1 (both halves of one hidden shard) and a single cluster has no gap
+    assert sharding.index_set_gaps(g["S_1112"]) == sharding.index_set_gaps(g["R_1"])
+    assert sharding.index_set_gaps([4, 5, 6])["min_gap"] == -1 and sharding.index_set_gaps([])["n_clusters"] == 0
+    # colluding CompNodes 1 and 2 pool {1,2,3,4,7,8,9,10,...}: clusters of 4, gaps of 2
+    union = g["R_1"] + g["R_2"]
+    assert sharding.index_set_gaps(union) == {"n_indices": 12, "n_clusters": 3, "min_gap": 2, "max_gap": 2}
+    for c, delta, n in [(2, 6, 18), (8, 64, 512), (3, 10, 100), (1, 5, 23), (8, 96, 1000)]:
+        r_of = sharding.cdelta_shard_of(n, c, delta)
+        for i in range(sharding.alpha_of(c, delta)):
+            held = np.flatnonzero(r_of == i)
+            gp = sharding.index_set_gaps(held)
+            if i >= delta // c:  # c does not divide delta: the last shard's clusters are cut to delta mod c tokens
+                assert gp["n_clusters"] < 2 or gp["min_gap"] == gp["max_gap"] == delta - delta % c
+                continue
+            if gp["n_clusters"] > 1:
+                assert gp["min_gap"] == gp["max_gap"] == delta - c == sharding.cluster_gap(c, delta) - 1
+            for rho in range(1, delta + 2):
+                if gp["n_clusters"] > 1:
+                    assert sharding.secure_hidden_state_criterion(held, rho) == (delta - c + 1 >= rho)
+                    assert sharding.secure_full_criterion(held, rho) == (delta - c + 1 >= rho + 1)
+
+
+def test_kl_gaps_follow_the_proof_of_the_theorem():
+    g = _golden()
+    r_of = sharding.cdelta_shard_of(18, 2, 6)
+    s_of = sharding.m_split_shard_of(r_of, 2)
+    R1 = [t - 1 for t in g["R_1"]]  # 0-based
+    # without m-split (S = R): between 2 and 7 (1-based) lie {3,4} of R_2 and {5,6} of R_3; R_1's own shard adds nothing
+    assert sharding.kl_gaps(R1, r_of, 3).tolist() == [-1, 2, 2]
+    # with the m = 2 split every foreign KV shard contributes one token per gap; R_1's own pieces none
+    assert sharding.kl_gaps(R1, s_of, 6).tolist() == [-1, -1, 1, 1, 1, 1]
+    # brute force over all index pairs on random sets
+    rng = np.random.default_rng(0)
+    for _ in range(50):
+        n = int(rng.integers(2, 30))
+        s_map = rng.integers(0, 3, n)
+        held = np.flatnonzero(rng.random(n) < 0.4)
+        got = sharding.kl_gaps(held, s_map, 3)
+        for k in range(3):
+            sizes = []
+            hs = sorted(held.tolist())
+            for a, b in zip(hs[:-1], hs[1:]):
+                cnt = sum(1 for t in range(a + 1, b) if s_map[t] == k)  # nothing between neighbours is held
+                if cnt:
+                    sizes.append(cnt)
+            assert got[k] == (min(sizes) if sizes else -1)
