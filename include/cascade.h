@@ -232,6 +232,54 @@ cascade_status_t cascade_attn_sharded_rope(const cascade_plan_t* plan, cascade_d
                                            void* stream);
 
 /*
+ * Shard-map generators and shard-safety measures.  HOST arrays only, integer only, no device work; the maps they
+ * write are what cascade_shard_plan takes.  Token indices are 0-based (the paper prints 1-based ones).
+ *
+ * cascade_cdelta_shard_map -- (c, delta)-sharding (Section 6, definition of a (c, delta)-sequence): sequence i holds
+ * the tokens i c .. i c + c - 1 of every period of delta tokens, shard_of[t] = (t mod delta) / c; the number of
+ * sequences that covers [N] is alpha = ceil(delta / c), written to *n_shards_out (optional).  If c does not divide
+ * delta the last sequence has clusters of delta mod c tokens.
+ *   shard_of  HOST int32 [n_tokens], written.   Errors: INVALID_ARG unless 1 <= c <= delta, n_tokens >= 0.
+ */
+cascade_status_t cascade_cdelta_shard_map(int32_t n_tokens, int32_t c, int32_t delta, int32_t* shard_of,
+                                          int32_t* n_shards_out);
+
+/*
+ * cascade_msplit_shard_map -- the m-split of AttnNodes (Section 6.4): every hidden shard R_i is cut into m pieces,
+ * R_{i,x} taking the members of sorted R_i at ranks x, x + m, x + 2m, ... (the rule the section's worked example
+ * with N = 18, c = 2, delta = 6, m = 2 follows), and the query/KV shards are S_{m i + x} = R_{i,x}; beta = m alpha.
+ *   r_shard_of  HOST int32 [n_tokens], values in [0, n_r_shards)     s_shard_of  HOST int32 [n_tokens], written
+ * Errors: INVALID_ARG (sizes, null arrays), BAD_MAP (an id outside [0, n_r_shards); the message names the token).
+ */
+cascade_status_t cascade_msplit_shard_map(int32_t n_tokens, const int32_t* r_shard_of, int32_t n_r_shards, int32_t m,
+                                          int32_t* s_shard_of);
+
+/*
+ * cascade_index_set_gaps -- clusters and gaps of the index set a node holds, or of the union a colluding set of nodes
+ * pools (CompNode_i: R_i; AttnNode_jk: S_j u T_k; appendix on collusion).  A cluster is a maximal run of consecutive
+ * held indices; the gap between neighbouring clusters is the number of indices strictly between them, i.e. the
+ * unknown tokens a generalized vocab-matching attack must enumerate (V^gap candidates).  For a (c, delta)-sequence
+ * every gap is delta - c (Section 6.2 states it as the cluster-to-cluster distance delta - c + 1).  Criteria:
+ *   Section 6.2 (leakage from the node's own hidden states):  min_gap + 1 >= rho
+ *   Theorem of Section 6.3 and the collusion appendix:         min_gap     >= rho
+ *   held  HOST uint8 [n_tokens], non-zero = the index is held.
+ *   n_indices, n_clusters, min_gap, max_gap: optional outputs; min_gap = max_gap = -1 with fewer than two clusters.
+ */
+cascade_status_t cascade_index_set_gaps(int32_t n_tokens, const uint8_t* held, int32_t* n_indices,
+                                        int32_t* n_clusters, int32_t* min_gap, int32_t* max_gap);
+
+/*
+ * cascade_kl_gaps -- the (k, l)-gaps from the proof of the Section 6.3 theorem: for the node's sorted indices
+ * r_1 < r_2 < ... and KV shard S_k, gap (k, l) = { s in S_k : r_l < s < r_{l+1} } without the node's own indices.
+ * The attack of the proof needs a NON-EMPTY gap with fewer than rho members, so the call reports, per KV shard, the
+ * size of the smallest non-empty gap over l (-1 if every gap of that shard is empty).
+ *   r_held  HOST uint8 [n_tokens]      s_shard_of  HOST int32 [n_tokens], values in [0, n_s_shards)
+ *   min_gap_per_shard  HOST int32 [n_s_shards], written.   Errors: INVALID_ARG, BAD_MAP.
+ */
+cascade_status_t cascade_kl_gaps(int32_t n_tokens, const uint8_t* r_held, const int32_t* s_shard_of,
+                                 int32_t n_s_shards, int32_t* min_gap_per_shard);
+
+/*
  * cascade_attn_decode_static -- the decode case of cascade_attn_sharded (one query row per sequence, bf16,
  * head_dim 128, n_heads / n_kv_heads in {1,2,4,8}) without a workspace argument and without any allocation.
  * (The paper has no counterpart: this is a convenience of this library, not a step of the method.)

@@ -29,6 +29,7 @@ EXPORTS = [
     "cascade_plan_get", "cascade_plan_dense_mask", "cascade_plan_device_status", "cascade_attn_partials",
     "cascade_merge", "cascade_attn_sharded", "cascade_workspace_bytes", "cascade_attn_decode_static",
     "cascade_kernel_timing_begin", "cascade_kernel_timing_end", "cascade_rope_table", "cascade_attn_sharded_rope",
+    "cascade_cdelta_shard_map", "cascade_msplit_shard_map", "cascade_index_set_gaps", "cascade_kl_gaps",
 ]
 
 
@@ -75,6 +76,11 @@ def lib() -> ctypes.CDLL:
         L.cascade_rope_table.argtypes = [i32, i32, ctypes.c_double, vp, vp]
         L.cascade_attn_sharded_rope.argtypes = [vp, i32, i32, i32, i32, i32, f32, vp, Strides, vp, Strides, vp, Strides,
                                                 vp, i32, vp, Strides, vp, vp, ctypes.c_size_t, vp]
+        pi32 = ctypes.POINTER(i32)
+        L.cascade_cdelta_shard_map.argtypes = [i32, i32, i32, vp, pi32]
+        L.cascade_msplit_shard_map.argtypes = [i32, vp, i32, i32, vp]
+        L.cascade_index_set_gaps.argtypes = [i32, vp, pi32, pi32, pi32, pi32]
+        L.cascade_kl_gaps.argtypes = [i32, vp, vp, i32, vp]
         L.cascade_kernel_timing_begin.argtypes = []
         L.cascade_kernel_timing_end.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
         for name in EXPORTS:
@@ -319,3 +325,41 @@ def cascade_attn_decode_static(plan: Plan, q: torch.Tensor, k: torch.Tensor, v: 
                                             k.data_ptr(), _strides(k), v.data_ptr(), _strides(v), o.data_ptr(),
                                             _strides(o), lse.data_ptr() if lse is not None else None, _stream()))
     return o, lse
+
+
+def _np_ptr(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def cascade_cdelta_shard_map(n_tokens: int, c: int, delta: int):
+    """(c, delta)-sharding: returns (shard_of int32 [n_tokens], alpha)."""
+    out = np.empty(n_tokens, np.int32)
+    alpha = ctypes.c_int32()
+    _check(lib().cascade_cdelta_shard_map(n_tokens, c, delta, _np_ptr(out), ctypes.byref(alpha)))
+    return out, alpha.value
+
+
+def cascade_msplit_shard_map(r_shard_of, n_r_shards: int, m: int) -> np.ndarray:
+    """m-split of hidden shards into query/KV shards S_{m i + x} = R_{i,x}."""
+    r = np.ascontiguousarray(r_shard_of, np.int32)
+    out = np.empty_like(r)
+    _check(lib().cascade_msplit_shard_map(r.shape[0], _np_ptr(r), n_r_shards, m, _np_ptr(out)))
+    return out
+
+
+def cascade_index_set_gaps(held) -> dict:
+    """Clusters and gaps of an index set given as membership flags over the tokens."""
+    h = np.ascontiguousarray(np.asarray(held) != 0, np.uint8)
+    vals = [ctypes.c_int32() for _ in range(4)]
+    _check(lib().cascade_index_set_gaps(h.shape[0], _np_ptr(h), *[ctypes.byref(v) for v in vals]))
+    return dict(zip(("n_indices", "n_clusters", "min_gap", "max_gap"), (v.value for v in vals)))
+
+
+def cascade_kl_gaps(r_held, s_shard_of, n_s_shards: int) -> np.ndarray:
+    """Smallest non-empty (k, l)-gap per KV shard for the node whose indices are flagged in r_held."""
+    h = np.ascontiguousarray(np.asarray(r_held) != 0, np.uint8)
+    s = np.ascontiguousarray(s_shard_of, np.int32)
+    assert h.shape == s.shape
+    out = np.empty(n_s_shards, np.int32)
+    _check(lib().cascade_kl_gaps(h.shape[0], _np_ptr(h), _np_ptr(s), n_s_shards, _np_ptr(out)))
+    return out
