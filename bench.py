@@ -319,6 +319,25 @@ def run_extras(torch, cb, wl, flush, peaks):
                         "frac_of_8tbs": gbs / 8000.0, "decode_plus_merge_ms": statistics.median(ms_f),
                         "decode_plus_merge_kv_gbs": w.kv_bytes() / (statistics.median(ms_f) * 1e-3) / 1e9}
     plan.destroy()
+    del q, k, v, o, parts, ws
+    # The shape of the paper's own latency tables: one BERT-Base layer's attention, 128-token prompt, bidirectional
+    # mask, fp32, (c, delta) = (8, 16) sharding over alpha = 2 nodes (launch-latency-bound at this size).
+    r_of, alpha = cb.cascade_cdelta_shard_map(128, 8, 16)
+    w = wl.make_workload("bert_base_n128", 1, 128, 128, 12, 12, 64, "f32", "round_robin", "round_robin", alpha, alpha,
+                         seed=5, causal=False)
+    q, k, v = _upload(w, torch, wl)
+    plan = cb.cascade_shard_plan(r_of, r_of, alpha, alpha, 0, False)
+    o = torch.empty_like(q)
+    ms_b = _time_steps(torch, lambda: cb.cascade_attn_sharded(plan, q, k, v, w.scale, out=o, want_lse=False), 20, 3,
+                       flush)
+    parts = cb.cascade_attn_partials(plan, q, k, v, w.scale)
+    ms_bp = _time_steps(torch, lambda: (cb.cascade_attn_partials(plan, q, k, v, w.scale, out=parts),
+                                        cb.cascade_merge(*parts, plan.dev_ptr("q_idx"), out=o, want_lse=False)), 20, 3,
+                        flush)
+    out["bert_base_n128_noncausal_f32"] = {"fused_ms": statistics.median(ms_b),
+                                           "partials_plus_merge_ms": statistics.median(ms_bp),
+                                           "sharding": "(c, delta) = (8, 16), alpha = 2"}
+    plan.destroy()
     return out
 
 
