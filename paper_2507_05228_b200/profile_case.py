@@ -3,7 +3,7 @@
     python -m paper_2507_05228_b200.profile_case <workload> <route> [--launches N] [--override k=v ...]
 
 workload: c1_tiny_f32 | c2_prefill_8b | c3_batched | c4_long_70b | c5_decode
-route:    fused | partials | merge | decode
+route:    fused | fused_rope | partials | merge | decode
 Prints the median CUDA-event time per launch (L2 flushed between launches).
 """
 from __future__ import annotations
@@ -21,7 +21,7 @@ from . import workloads as wl
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("workload")
-    ap.add_argument("route", choices=["fused", "partials", "merge", "decode"])
+    ap.add_argument("route", choices=["fused", "fused_rope", "partials", "merge", "decode"])
     ap.add_argument("--launches", type=int, default=3)
     ap.add_argument("--override", nargs="*", default=[])
     args = ap.parse_args()
@@ -44,7 +44,10 @@ def main():
         ws = torch.empty(max(nb, 1), dtype=torch.uint8, device="cuda")
     if args.route in ("partials", "merge", "decode"):
         parts = cb.cascade_attn_partials(plan, q, k, v, w.scale, workspace=ws)
+    table = cb.cascade_rope_table(max(w.q_pos_offset + w.n_q, w.n_kv), w.d, 500000.0) if args.route == "fused_rope" else None
     fn = {
+        "fused_rope": lambda: cb.cascade_attn_sharded_rope(plan, q, k, v, w.scale, table, out=o, want_lse=False,
+                                                           workspace=ws),
         "fused": lambda: cb.cascade_attn_sharded(plan, q, k, v, w.scale, out=o, want_lse=False, workspace=ws),
         "partials": lambda: cb.cascade_attn_partials(plan, q, k, v, w.scale, out=parts, workspace=ws),
         "decode": lambda: cb.cascade_attn_partials(plan, q, k, v, w.scale, out=parts),
