@@ -806,6 +806,10 @@ if constexpr (kRope) {
         const bool leader = elect_one();
         ChunkCursor cur;
         cur.start(tab, n_act);
+        // The shard-major copies are written by the gather grid launched just before this one; when this grid was
+        // launched as its programmatic dependent it may have started early, so wait here for that grid to complete
+        // (a no-op otherwise).  Nothing else in this kernel reads what the gather grid writes.
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         for (int i = 0; i < n_tiles; ++i) {
           const int nch = tile_chunks(i);
           const int st = i % n_stages;
@@ -895,9 +899,21 @@ cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void
                                        (p.os.head * 2) % 32 == 0
                                  : a32(p.o_part);
   TimedLaunch timed(stream);
-  kernel<<<(unsigned)n_ctas, tc::kThreads, tc::kSmemBytes, stream>>>(p, lg, tile_major, wide_store, tma);
+  // Programmatic dependent launch on the gather grid that precedes it in the stream: the set-up of the CTAs overlaps
+  // the gather's tail.  Not while kernel timing is recording: the event between the two launches must separate them.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)n_ctas);
+  cfg.blockDim = dim3(tc::kThreads);
+  cfg.dynamicSmemBytes = tc::kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = timing_recording() ? 0 : 1;
+  e = cudaLaunchKernelEx(&cfg, kernel, p, lg, tile_major, wide_store, tma);
   count_launch();
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace cascade

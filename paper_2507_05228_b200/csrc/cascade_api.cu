@@ -29,6 +29,8 @@ static std::vector<cudaEvent_t> g_ev_start, g_ev_stop;
 static size_t g_timed = 0;  // launches bracketed since begin
 constexpr size_t kMaxTimedLaunches = 8192;
 
+bool timing_recording() { return g_timing_on; }
+
 void timing_mark(cudaStream_t stream, bool start) {
   if (!g_timing_on) return;
   if (start) {

@@ -87,6 +87,7 @@ void set_error(const char* fmt, ...);
 void count_launch(int n = 1);
 // Kernel timing (cascade_kernel_timing_begin / _end): brackets a launch with events when recording is on.
 void timing_mark(cudaStream_t stream, bool start);
+bool timing_recording();  // true between cascade_kernel_timing_begin and _end
 struct TimedLaunch {  // RAII: events around the launches issued while it lives
   cudaStream_t st;
   explicit TimedLaunch(cudaStream_t s) : st(s) { timing_mark(st, true); }

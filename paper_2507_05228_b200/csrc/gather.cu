@@ -13,6 +13,9 @@ constexpr int kGatherRowsPerCta = 64;
 
 __global__ void __launch_bounds__(256) gather_kv_kernel(AttnParams p, __nv_bfloat16* k_out, __nv_bfloat16* v_out) {
   constexpr int D = 128;
+  // The attention kernel that follows may be launched as a programmatic dependent: its CTAs may start their set-up
+  // (query loads, shard tables, TMEM) now; they wait for this grid to finish before they touch the copies.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const PlanDev& pl = p.plan;
   const int g = blockIdx.y, b = blockIdx.z;
   const int map = pl.n_maps == 1 ? 0 : b;
@@ -64,6 +67,7 @@ __device__ __forceinline__ void rotate8(uint4& lo, uint4& hi, const float2* __re
 __global__ void __launch_bounds__(256) gather_kv_rope_kernel(AttnParams p, __nv_bfloat16* k_out, __nv_bfloat16* v_out) {
   constexpr int D = 128;
   constexpr int kPasses = kGatherRowsPerCta / 32;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // as in gather_kv_kernel
   const PlanDev& pl = p.plan;
   const int g = blockIdx.y, b = blockIdx.z;
   const int map = pl.n_maps == 1 ? 0 : b;
