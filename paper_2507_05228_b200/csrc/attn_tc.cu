@@ -55,12 +55,14 @@ constexpr int kRegsOther = 72;
 constexpr int kChunk = 32;                // keys per chunk of the KV stream
 constexpr int kChunkBytes = kChunk * 128; // one 64-column half of a chunk in a tile
 constexpr int kMaxShards = 256;           // KV shards per CTA whose bookkeeping fits in shared memory
+constexpr int kStageRowBytes = 272;       // output rows staged for the bulk copies: 256 bytes + 16 of padding
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int kOffQ = 0;
 constexpr int kOffK = kOffQ + 2 * kTileBytes;
 constexpr int kOffV = kOffK + kKStages * kTileBytes;
 constexpr int kOffBar = kOffV + kVStages * kTileBytes;
+static_assert(2 * kM * kStageRowBytes <= kOffV, "the output staging area must fit in the Q and K tiles");
 constexpr int kNumBars = 24;
 constexpr int kOffMisc = kOffBar + kNumBars * 8;   // tmem slot, abort flag, 12 progress words
 constexpr int kOffShard = kOffMisc + 64;           // int32 [5][kMaxShards], see ShardTab
@@ -269,12 +271,6 @@ __device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
-// 32-byte store: one full sector per lane (rows of the output are written by one thread each)
-__device__ __forceinline__ void st_global_v8(void* ptr, const uint32_t (&v)[8]) {
-  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(ptr), "r"(v[0]), "r"(v[1]), "r"(v[2]),
-               "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
-               : "memory");
-}
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&h);
@@ -313,7 +309,7 @@ struct TmaArgs {
 // were turned by the gather pass), Algorithm 2.
 template <bool kRope>
 __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_constant__ AttnParams p, int lg,
-                                                              int tile_major, int wide_store,
+                                                              int tile_major,
                                                               const __grid_constant__ TmaArgs tma) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -662,6 +658,20 @@ if constexpr (kRope) {
       }
       note(8 * n_tiles + 3);
       // ---- epilogue
+      // Where this row goes is looked up before the wait for the last product, which hides the load.
+      __nv_bfloat16* dst = nullptr;
+      int64_t stat = 0;
+      if (row_ok) {
+        if (p.fused) {
+          const int tok = __ldg(q_idx + slot);
+          stat = ((int64_t)b * pl.n_q + tok) * p.H + head;
+          dst = static_cast<__nv_bfloat16*>(p.o_out) + (int64_t)b * p.os.batch + (int64_t)tok * p.os.token +
+                (int64_t)head * p.os.head;
+        } else {
+          stat = (((int64_t)b * P + part) * pl.n_q + slot) * p.H + head;
+          dst = static_cast<__nv_bfloat16*>(p.o_part) + stat * kD;
+        }
+      }
       float o_scale = 0.f, m_out = -INFINITY, l_out = 0.f;
       if (n_tiles > 0) {
         wait_bar(wc, bar(O_FULL), 0u, 3, n_tiles);
@@ -672,21 +682,18 @@ if constexpr (kRope) {
           m_out = m_true * 0.6931471805599453f;   // natural-log units
         }
       }
-      __nv_bfloat16* dst = nullptr;
       if (row_ok) {
         if (p.fused) {
-          const int tok = __ldg(q_idx + slot);
-          dst = static_cast<__nv_bfloat16*>(p.o_out) + (int64_t)b * p.os.batch + (int64_t)tok * p.os.token +
-                (int64_t)head * p.os.head;
-          if (p.lse_out)
-            p.lse_out[((int64_t)b * pl.n_q + tok) * p.H + head] = l_out > 0.f ? m_out + logf(l_out) : -INFINITY;
+          if (p.lse_out) p.lse_out[stat] = l_out > 0.f ? m_out + logf(l_out) : -INFINITY;
         } else {
-          const int64_t stat = (((int64_t)b * P + part) * pl.n_q + slot) * p.H + head;
-          dst = static_cast<__nv_bfloat16*>(p.o_part) + stat * kD;
           p.m_part[stat] = m_out;
           p.l_part[stat] = l_out;
         }
       }
+      // Every product of the CTA has completed, so the Q / K tiles in shared memory are free: the thread stages its
+      // 256-byte output row there (rows 272 bytes apart, which spreads a warp's 16-byte stores over all banks) and hands
+      // it to the copy engine as one bulk copy, instead of writing 32-byte pieces of 32 different rows per instruction.
+      uint8_t* stage = smem + kOffQ + (s * kM + m) * kStageRowBytes;
 #pragma unroll
       for (int cc = 0; cc < 4; ++cc) {
         uint32_t o[32];
@@ -697,21 +704,22 @@ if constexpr (kRope) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) o[j] = 0u;
         }
-        if (row_ok) {
 #pragma unroll
-          for (int j = 0; j < 32; j += 16) {
-            uint32_t val[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e)
-              val[e] = pack_bf16x2(__uint_as_float(o[j + 2 * e]) * o_scale, __uint_as_float(o[j + 2 * e + 1]) * o_scale);
-            if (wide_store) {
-              st_global_v8(dst + cc * 32 + j, val);
-            } else {
-              *reinterpret_cast<uint4*>(dst + cc * 32 + j) = make_uint4(val[0], val[1], val[2], val[3]);
-              *reinterpret_cast<uint4*>(dst + cc * 32 + j + 8) = make_uint4(val[4], val[5], val[6], val[7]);
-            }
-          }
+        for (int j = 0; j < 32; j += 8) {
+          uint4 val;
+          val.x = pack_bf16x2(__uint_as_float(o[j]) * o_scale, __uint_as_float(o[j + 1]) * o_scale);
+          val.y = pack_bf16x2(__uint_as_float(o[j + 2]) * o_scale, __uint_as_float(o[j + 3]) * o_scale);
+          val.z = pack_bf16x2(__uint_as_float(o[j + 4]) * o_scale, __uint_as_float(o[j + 5]) * o_scale);
+          val.w = pack_bf16x2(__uint_as_float(o[j + 6]) * o_scale, __uint_as_float(o[j + 7]) * o_scale);
+          *reinterpret_cast<uint4*>(stage + cc * 64 + j * 2) = val;
         }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // this thread's writes -> the copy engine's reads
+      if (row_ok) {
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], 256;" ::"l"(dst), "r"(smem_u32(stage))
+                     : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // the row has left shared memory
       }
       tc_fence_before();
     }
@@ -893,11 +901,6 @@ cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void
   const int64_t n_ctas = (int64_t)p.plan.n_qtiles[3 - lg] * (p.H >> lg) * p.batch * n_parts;
   if (n_ctas >= (int64_t)1 << 31) return cudaErrorInvalidConfiguration;
   const int tile_major = n_ctas <= 8 * 148;  // few CTAs per SM: balance matters more than L2 locality
-  // 32-byte stores of the output rows need 32-byte aligned rows (the interface only asks for 16)
-  const auto a32 = [](const void* ptr) { return ((uintptr_t)ptr & 31) == 0; };
-  const int wide_store = p.fused ? a32(p.o_out) && (p.os.batch * 2) % 32 == 0 && (p.os.token * 2) % 32 == 0 &&
-                                       (p.os.head * 2) % 32 == 0
-                                 : a32(p.o_part);
   TimedLaunch timed(stream);
   // Programmatic dependent launch on the gather grid that precedes it in the stream: the set-up of the CTAs overlaps
   // the gather's tail.  Not while kernel timing is recording: the event between the two launches must separate them.
@@ -911,7 +914,7 @@ cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = timing_recording() ? 0 : 1;
-  e = cudaLaunchKernelEx(&cfg, kernel, p, lg, tile_major, wide_store, tma);
+  e = cudaLaunchKernelEx(&cfg, kernel, p, lg, tile_major, tma);
   count_launch();
   return e;
 }

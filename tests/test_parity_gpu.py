@@ -186,7 +186,7 @@ def test_tensor_core_route_workspace_contract_and_unaligned_output(gu):
         with pytest.raises(cb.CascadeError) as ei:
             call(plan, q, k, v, w.scale, workspace=small)
         assert ei.value.status == 4
-    # an output whose rows are 16- but not 32-byte aligned takes the narrow-store epilogue
+    # an output whose rows are 16- but not 32-byte aligned (the interface asks for 16; the row copies need no more)
     flat = torch.zeros(q.numel() + 8, dtype=torch.bfloat16, device="cuda")
     o_view = flat[8:].view(q.shape)
     assert o_view.data_ptr() % 32 == 16
