@@ -17,7 +17,9 @@
 //   0-3   softmax of sub-tile 0, 4-7 softmax of sub-tile 1: thread = MMA row = TMEM lane.  Reads the logits S with
 //         tcgen05.ld, applies the shard mask (the row sees the first vis[slot][k] keys of the shard), keeps the running
 //         max / sum, writes the probabilities P as bf16 back into the TMEM columns of S, rescales the output
-//         accumulator in TMEM when the running max moved by more than 2^8, and runs the epilogue.
+//         accumulator in TMEM when the running max moved by more than 2^8, and runs the epilogue: the scaled output
+//         row goes through shared memory (the Q / K tiles are free by then) to the copy engine, one 256-byte bulk
+//         copy per row.
 //   8     MMA issuer: S_s = Q_s K^T (operands in shared memory) and O_s += P_s V (P from TMEM), issued as
 //         PV_0(i), QK_0(i+1), PV_1(i), QK_1(i+1) so that the tensor pipe works on one sub-tile while the other is in
 //         its softmax.  QK_s(i+1) overwrites the columns PV_s(i) reads P from; MMAs execute in issue order, which
@@ -30,7 +32,10 @@
 //         the caller's tensors was far too slow for the K/V stream (measured: one 512-byte TMA row gather per ~36
 //         cycles per SM; 16-byte cp.async: one 512-byte request per ~90 cycles per warp).  The two query
 //         sub-tiles are gathered once per CTA by the softmax threads themselves (plain 16-byte loads).
-//   11    idle (keeps the register-reallocation groups of four warps whole).
+//   11    builds the table of the shards the CTA sees anything of (what each role needs per shard, and the number of
+//         chunks), then idles; it also keeps the register-reallocation groups of four warps whole.
+// The grid is launched as a programmatic dependent of the gather grid: everything up to the loaders' first TMA load
+// may run while the gather is still writing the shard-major copies (the loaders wait with griddepcontrol.wait).
 // Every mbarrier wait is bounded: on expiry the CTA raises a flag, records a code in the plan's status word
 // and drains without waiting again.
 #include <cuda.h>
