@@ -280,6 +280,27 @@ cascade_status_t cascade_kl_gaps(int32_t n_tokens, const uint8_t* r_held, const 
                                  int32_t n_s_shards, int32_t* min_gap_per_shard);
 
 /*
+ * cascade_attn_sharded_host -- cascade_attn_sharded for callers whose tensors live in HOST memory (the paper's nodes
+ * exchange q, k, v and the outputs over a network; here the host side of the PCIe link stands in for it).  The call
+ * copies k and v to the device, then works through the KV heads one at a time: the G = n_heads / n_kv_heads query
+ * heads of KV head g are uploaded on one copy stream while the fused attention of head g - 1 runs on the caller's
+ * stream and the output of head g - 2 travels back on a second copy stream, so the transfers in both directions
+ * overlap each other and the compute.  Results are those of cascade_attn_sharded.
+ *   q_host, o_host  HOST, dense [batch][n_q][n_heads][head_dim]; k_host, v_host  HOST, dense
+ *                   [batch][n_kv][n_kv_heads][head_dim].  Pinned memory is needed for the copies to be asynchronous.
+ *   workspace       DEVICE, 256-byte aligned, cascade_workspace_bytes(CASCADE_CALL_SHARDED_HOST) bytes: staging for
+ *                   q, k, v, o and the scratch of one head group.  Overwritten by every call.
+ * All work is ordered after what `stream` holds at the time of the call, and `stream` waits for the last output
+ * copy: synchronising `stream` makes o_host valid.  The first call on a device creates two internal copy streams and
+ * their events (no device memory).  Errors as cascade_attn_sharded, plus CASCADE_ERR_INVALID_ARG for more than 128 KV
+ * heads.
+ */
+cascade_status_t cascade_attn_sharded_host(const cascade_plan_t* plan, cascade_dtype_t dtype, int32_t batch,
+                                           int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, float scale,
+                                           const void* q_host, const void* k_host, const void* v_host,
+                                           void* o_host, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * cascade_attn_decode_static -- the decode case of cascade_attn_sharded (one query row per sequence, bf16,
  * head_dim 128, n_heads / n_kv_heads in {1,2,4,8}) without a workspace argument and without any allocation.
  * (The paper has no counterpart: this is a convenience of this library, not a step of the method.)
@@ -307,7 +328,7 @@ cascade_status_t cascade_attn_decode_static(const cascade_plan_t* plan, int32_t 
                                             cascade_strides_t v_strides, void* o_out, cascade_strides_t o_strides,
                                             float* lse_out, void* stream);
 
-enum { CASCADE_CALL_PARTIALS = 0, CASCADE_CALL_SHARDED = 1 };
+enum { CASCADE_CALL_PARTIALS = 0, CASCADE_CALL_SHARDED = 1, CASCADE_CALL_SHARDED_HOST = 2 };
 
 /* Scratch bytes the given call needs for this plan and shape (0 if none).  The workspace must be
  * 256-byte aligned. */

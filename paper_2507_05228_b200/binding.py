@@ -30,6 +30,7 @@ EXPORTS = [
     "cascade_merge", "cascade_attn_sharded", "cascade_workspace_bytes", "cascade_attn_decode_static",
     "cascade_kernel_timing_begin", "cascade_kernel_timing_end", "cascade_rope_table", "cascade_attn_sharded_rope",
     "cascade_cdelta_shard_map", "cascade_msplit_shard_map", "cascade_index_set_gaps", "cascade_kl_gaps",
+    "cascade_attn_sharded_host",
 ]
 
 
@@ -81,6 +82,7 @@ def lib() -> ctypes.CDLL:
         L.cascade_msplit_shard_map.argtypes = [i32, vp, i32, i32, vp]
         L.cascade_index_set_gaps.argtypes = [i32, vp, pi32, pi32, pi32, pi32]
         L.cascade_kl_gaps.argtypes = [i32, vp, vp, i32, vp]
+        L.cascade_attn_sharded_host.argtypes = [vp, i32, i32, i32, i32, i32, f32, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.cascade_kernel_timing_begin.argtypes = []
         L.cascade_kernel_timing_end.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
         for name in EXPORTS:
@@ -310,6 +312,27 @@ def cascade_attn_sharded_rope(plan: Plan, q: torch.Tensor, k: torch.Tensor, v: t
                                            rope_table.data_ptr(), rope_table.shape[0], o.data_ptr(), _strides(o),
                                            lse.data_ptr() if lse is not None else None, ws_ptr, ws_bytes, _stream()))
     return o, lse
+
+
+CALL_SHARDED_HOST = 2
+
+
+def cascade_attn_sharded_host(plan: Plan, q_host: torch.Tensor, k_host: torch.Tensor, v_host: torch.Tensor,
+                              scale: float, out_host: torch.Tensor, workspace: torch.Tensor):
+    """Fused attention on dense HOST tensors (pinned for asynchronous copies): uploads, computes and downloads one KV
+    head group after another with the three overlapped.  `workspace` is a device uint8 tensor of
+    cascade_workspace_bytes(plan, CALL_SHARDED_HOST, ...) bytes.  Returns out_host; synchronise the current stream
+    before reading it."""
+    B, n_q, H, d = q_host.shape
+    Hkv = k_host.shape[2]
+    code = _dtype_code(q_host)
+    for t in (q_host, k_host, v_host, out_host):
+        assert not t.is_cuda and t.is_contiguous(), "dense host tensors expected"
+    assert workspace.is_cuda and workspace.dtype == torch.uint8
+    _check(lib().cascade_attn_sharded_host(plan.handle, code, B, H, Hkv, d, scale, q_host.data_ptr(),
+                                           k_host.data_ptr(), v_host.data_ptr(), out_host.data_ptr(),
+                                           workspace.data_ptr(), workspace.numel(), _stream()))
+    return out_host
 
 
 def cascade_attn_decode_static(plan: Plan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, scale: float, out=None,

@@ -25,6 +25,7 @@ void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 // ---- kernel timing
 static bool g_timing_on = false;
+constexpr int kMaxHostGroups = 128;  // head groups cascade_attn_sharded_host pipelines over
 static std::vector<cudaEvent_t> g_ev_start, g_ev_stop;
 static size_t g_timed = 0;  // launches bracketed since begin
 constexpr size_t kMaxTimedLaunches = 8192;
@@ -503,6 +504,50 @@ static cascade_status_t run_tc(const AttnParams& p, const char* fn, const cascad
   return CASCADE_OK;
 }
 
+// How many KV heads cascade_attn_sharded_host moves and computes at a time: enough that a strided row of the group's
+// query heads is at least 2 KiB (narrower rows make the 2-D copies slow), at most all of them.
+static int host_call_group(int H, int Hkv, int d, size_t es) {
+  const size_t row = (size_t)(H / Hkv) * d * es;
+  int gs = 1;
+  while (gs < Hkv && row * gs < 2048) ++gs;
+  while (Hkv % gs != 0) ++gs;
+  return gs;
+}
+
+// Device-side staging of cascade_attn_sharded_host: dense copies of q, k, v, o and the scratch of one head group's
+// fused call, each region 256-byte aligned.
+struct HostCallLayout {
+  size_t q, k, v, o, inner, inner_bytes, total;
+};
+static HostCallLayout host_call_layout(const cascade_plan_t* plan, cascade_dtype_t dtype, int batch, int H, int Hkv,
+                                       int d) {
+  const size_t es = elt_size(dtype);
+  const size_t q_bytes = (size_t)batch * plan->dev.n_q * H * d * es;
+  const size_t kv_bytes = (size_t)batch * plan->dev.n_kv * Hkv * d * es;
+  const int G = H / Hkv, gs = host_call_group(H, Hkv, d, es);
+  HostCallLayout L;
+  L.q = 0;
+  L.k = L.q + align_up(q_bytes, 256);
+  L.v = L.k + align_up(kv_bytes, 256);
+  L.o = L.v + align_up(kv_bytes, 256);
+  L.inner = L.o + align_up(q_bytes, 256);
+  // gs KV heads and their query heads per inner call
+  const bool decode = use_decode(plan, dtype, G * gs, gs, d);
+  L.inner_bytes = decode ? decode_ws_bytes(plan, dtype, batch, G * gs, d)
+                         : (use_tc(plan, dtype, d) ? 2 * sorted_kv_bytes(plan, batch, gs) : 0);
+  L.total = L.inner + align_up(L.inner_bytes, 256);
+  return L;
+}
+
+// Copy streams and events of cascade_attn_sharded_host, made on first use per device.
+struct HostCallStreams {
+  bool ready = false;
+  cudaStream_t h2d = nullptr, d2h = nullptr;
+  cudaEvent_t start = nullptr, done = nullptr;
+  cudaEvent_t uploaded[kMaxHostGroups], computed[kMaxHostGroups];
+};
+static HostCallStreams g_host_streams[16];
+
 }  // namespace cascade
 
 extern "C" {
@@ -524,6 +569,8 @@ cascade_status_t cascade_workspace_bytes(const cascade_plan_t* plan, int32_t whi
     *out_bytes = tc_bytes;
   } else if (which_call == CASCADE_CALL_SHARDED) {
     *out_bytes = decode ? decode_ws_bytes(plan, dtype, batch, n_heads, head_dim) : tc_bytes;
+  } else if (which_call == CASCADE_CALL_SHARDED_HOST) {
+    *out_bytes = host_call_layout(plan, dtype, batch, n_heads, n_kv_heads, head_dim).total;
   } else {
     set_error("cascade_workspace_bytes: unknown call %d", which_call);
     return CASCADE_ERR_INVALID_ARG;
@@ -741,6 +788,102 @@ cascade_status_t cascade_rope_table(int32_t n_positions, int32_t head_dim, doubl
   cudaError_t e = launch_rope_table(n_positions, head_dim, base, reinterpret_cast<float2*>(table),
                                     (cudaStream_t)stream);
   if (e != cudaSuccess) return cuda_fail(e, "cascade_rope_table: launch");
+  return CASCADE_OK;
+}
+
+cascade_status_t cascade_attn_sharded_host(const cascade_plan_t* plan, cascade_dtype_t dtype, int32_t batch,
+                                           int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, float scale,
+                                           const void* q_host, const void* k_host, const void* v_host, void* o_host,
+                                           void* workspace, size_t workspace_bytes, void* stream) {
+  const char* fn = "cascade_attn_sharded_host";
+  if (!plan || !q_host || !k_host || !v_host || !o_host) {
+    set_error("%s: null pointer", fn);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (!plan->dev_blob) {
+    set_error("%s: the plan was built by cascade_shard_plan_host and has no device arrays", fn);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (dtype != CASCADE_F32 && dtype != CASCADE_BF16) {
+    set_error("%s: unknown dtype %d", fn, (int)dtype);
+    return CASCADE_ERR_UNSUPPORTED;
+  }
+  if (batch < 1 || n_heads < 1 || n_kv_heads < 1 || n_heads % n_kv_heads != 0 || n_kv_heads > kMaxHostGroups) {
+    set_error("%s: bad batch or head counts (at most %d KV heads)", fn, kMaxHostGroups);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (head_dim != 64 && head_dim != 128) {
+    set_error("%s: head_dim %d unsupported (64 or 128)", fn, head_dim);
+    return CASCADE_ERR_UNSUPPORTED;
+  }
+  const HostCallLayout L = host_call_layout(plan, dtype, batch, n_heads, n_kv_heads, head_dim);
+  if (!workspace || workspace_bytes < L.total || ((uintptr_t)workspace & 255)) {
+    set_error("%s: workspace of %zu bytes (256-byte aligned) required, got %zu", fn, L.total, workspace_bytes);
+    return CASCADE_ERR_WORKSPACE;
+  }
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_sharded_host: cudaGetDevice");
+  if (dev < 0 || dev >= 16) {
+    set_error("%s: device ordinal %d not supported", fn, dev);
+    return CASCADE_ERR_UNSUPPORTED;
+  }
+  HostCallStreams& hs = g_host_streams[dev];
+  if (!hs.ready) {
+    e = cudaStreamCreateWithFlags(&hs.h2d, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&hs.d2h, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&hs.start, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&hs.done, cudaEventDisableTiming);
+    for (int g = 0; g < kMaxHostGroups && e == cudaSuccess; ++g) {
+      e = cudaEventCreateWithFlags(&hs.uploaded[g], cudaEventDisableTiming);
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&hs.computed[g], cudaEventDisableTiming);
+    }
+    if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_sharded_host: creating streams and events");
+    hs.ready = true;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  char* ws = (char*)workspace;
+  const size_t es = elt_size(dtype);
+  const int G = n_heads / n_kv_heads;
+  const int gs = host_call_group(n_heads, n_kv_heads, head_dim, es);  // KV heads per group
+  const size_t q_rows = (size_t)batch * plan->dev.n_q, kv_rows = (size_t)batch * plan->dev.n_kv;
+  const size_t q_pitch = (size_t)n_heads * head_dim * es, kv_pitch = (size_t)n_kv_heads * head_dim * es;
+  const size_t q_width = (size_t)gs * G * head_dim * es;  // the query heads of one group, contiguous in a token row
+  const cascade_strides_t qs = {(int64_t)plan->dev.n_q * n_heads * head_dim, (int64_t)n_heads * head_dim, head_dim};
+  const cascade_strides_t ks = {(int64_t)plan->dev.n_kv * n_kv_heads * head_dim, (int64_t)n_kv_heads * head_dim,
+                                head_dim};
+  // the copy streams start after whatever the caller's stream has queued (it may still use the workspace)
+  e = cudaEventRecord(hs.start, st);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(hs.h2d, hs.start, 0);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(hs.d2h, hs.start, 0);
+  // K and V are small next to Q and O and contiguous: one copy each, up front (per-head copies of 256-byte rows were
+  // measured slower than the pipelining gains)
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ws + L.k, k_host, kv_rows * kv_pitch, cudaMemcpyHostToDevice, hs.h2d);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ws + L.v, v_host, kv_rows * kv_pitch, cudaMemcpyHostToDevice, hs.h2d);
+  if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_sharded_host: queuing the K/V copies");
+  for (int g = 0; g < n_kv_heads / gs; ++g) {
+    const size_t q_off = (size_t)g * q_width, kv_off = (size_t)g * gs * head_dim * es;
+    e = cudaMemcpy2DAsync(ws + L.q + q_off, q_pitch, (const char*)q_host + q_off, q_pitch, q_width, q_rows,
+                          cudaMemcpyHostToDevice, hs.h2d);
+    if (e == cudaSuccess) e = cudaEventRecord(hs.uploaded[g], hs.h2d);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(st, hs.uploaded[g], 0);
+    if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_sharded_host: queuing a query copy");
+    cascade_status_t rc = attn_sharded_impl(fn, plan, dtype, batch, G * gs, gs, head_dim, scale, ws + L.q + q_off, qs,
+                                            ws + L.k + kv_off, ks, ws + L.v + kv_off, ks, nullptr, 0,
+                                            ws + L.o + q_off, qs, nullptr, L.inner_bytes ? ws + L.inner : nullptr,
+                                            L.inner_bytes, st);
+    if (rc != CASCADE_OK) return rc;
+    e = cudaEventRecord(hs.computed[g], st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(hs.d2h, hs.computed[g], 0);
+    if (e == cudaSuccess)
+      e = cudaMemcpy2DAsync((char*)o_host + q_off, q_pitch, ws + L.o + q_off, q_pitch, q_width, q_rows,
+                            cudaMemcpyDeviceToHost, hs.d2h);
+    if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_sharded_host: queuing an output copy");
+  }
+  // the caller's stream is done when the last output copy is
+  e = cudaEventRecord(hs.done, hs.d2h);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(st, hs.done, 0);
+  if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_sharded_host: joining the copy stream");
   return CASCADE_OK;
 }
 
