@@ -505,11 +505,12 @@ static cascade_status_t run_tc(const AttnParams& p, const char* fn, const cascad
 }
 
 // How many KV heads cascade_attn_sharded_host moves and computes at a time: enough that a strided row of the group's
-// query heads is at least 2 KiB (narrower rows make the 2-D copies slow), at most all of them.
+// query heads is at least 1 KiB (256-byte rows made the 2-D copies slower than the pipelining gained; 2 KiB rows, i.e.
+// half as many stages, were slower again: 0.80 / 0.66 / 0.72 ms on the headline shape), at most all of them.
 static int host_call_group(int H, int Hkv, int d, size_t es) {
   const size_t row = (size_t)(H / Hkv) * d * es;
   int gs = 1;
-  while (gs < Hkv && row * gs < 2048) ++gs;
+  while (gs < Hkv && row * gs < 1024) ++gs;
   while (Hkv % gs != 0) ++gs;
   return gs;
 }
