@@ -346,10 +346,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
     hg = rem % n_hg;
     bz = rem / n_hg;
   } else {
-    const int rem = blockIdx.x / n_qt;
-    tile_idx = blockIdx.x % n_qt;
+    // the KV shards of one query tile (partials) are neighbours, so that its rows are read from HBM once and the
+    // CTAs running at a time walk all shards of one KV head
+    const int rem = blockIdx.x / (n_qt * n_parts);
+    tile_idx = (blockIdx.x / n_parts) % n_qt;
     hg = rem % n_hg;
-    bz = rem / n_hg;
+    bz = (rem / n_hg) * n_parts + blockIdx.x % n_parts;
   }
   const int b = bz / n_parts;
   const int part = bz % n_parts;
