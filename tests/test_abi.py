@@ -72,7 +72,16 @@ def test_host_side_argument_checks(binding):
     rc = L.cascade_attn_partials(plan.handle, 1, 1, 1, 1, 128, 1.0, 256, S4, 256, S4, 256, S4, 256, 256, 256,
                                  None, 0, None)
     assert rc == 1 and b"cascade_shard_plan_host" in L.cascade_last_error()
+    # the host-buffer call refuses null pointers and a host-only plan before touching CUDA; its workspace size is
+    # staging for q, k, v, o plus one head group's scratch
+    hb = np.zeros(16, np.uint8).ctypes.data_as(ctypes.c_void_p)
+    assert L.cascade_attn_sharded_host(plan.handle, 1, 1, 4, 2, 128, 1.0, None, hb, hb, hb, hb, 0, None) == 1
+    assert L.cascade_attn_sharded_host(plan.handle, 1, 1, 4, 2, 128, 1.0, hb, hb, hb, hb, hb, 0, None) == 1
+    assert b"cascade_shard_plan_host" in L.cascade_last_error()
     nbytes = ctypes.c_size_t()
+    assert L.cascade_workspace_bytes(plan.handle, 2, 1, 1, 4, 2, 128, ctypes.byref(nbytes)) == 0
+    q_b, kv_b = 8 * 4 * 128 * 2, 8 * 2 * 128 * 2
+    assert nbytes.value >= 2 * q_b + 2 * kv_b and nbytes.value % 256 == 0
     assert L.cascade_workspace_bytes(plan.handle, 0, 1, 1, 4, 3, 128, ctypes.byref(nbytes)) == 1
     assert L.cascade_workspace_bytes(plan.handle, 9, 1, 1, 4, 2, 128, ctypes.byref(nbytes)) == 1
     plan.destroy()
