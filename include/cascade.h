@@ -301,6 +301,21 @@ cascade_status_t cascade_attn_sharded_host(const cascade_plan_t* plan, cascade_d
                                            void* o_host, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * cascade_plan_advance -- moves the query block of a plan to a new position: token-sharded KV caching (Appendix F,
+ * "Caching").  Under a (c, delta)-style scheme the shard of every future token is known in advance, so a decode loop
+ * builds ONE plan over the whole cache capacity (n_kv = capacity, every slot already mapped to its KV shard, n_q = 1)
+ * and, for each generated token, writes that token's k and v rows at its index of the caller's cache tensors and
+ * calls this function with the token's position: the causal mask (key token <= query position) then admits exactly
+ * the cache rows written so far, and the new row belongs to its shard's list without any list being rebuilt.
+ * Recomputes VIS and PAIR_CLASS for query position q_pos_offset + token index (host arrays at once, device arrays in
+ * stream order); the index lists do not change.  Works for any n_q (a prefill chunk that slides along the sequence);
+ * the work-sorted order of the plan's query tiles is left as it was built, which affects speed only.
+ * Calls that use the plan before and after must be on `stream` or ordered with it.
+ * Errors: CASCADE_ERR_INVALID_ARG (null plan), CASCADE_ERR_CUDA.
+ */
+cascade_status_t cascade_plan_advance(cascade_plan_t* plan, int32_t q_pos_offset, void* stream);
+
+/*
  * cascade_attn_decode_static -- the decode case of cascade_attn_sharded (one query row per sequence, bf16,
  * head_dim 128, n_heads / n_kv_heads in {1,2,4,8}) without a workspace argument and without any allocation.
  * (The paper has no counterpart: this is a convenience of this library, not a step of the method.)

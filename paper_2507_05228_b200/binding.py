@@ -30,7 +30,7 @@ EXPORTS = [
     "cascade_merge", "cascade_attn_sharded", "cascade_workspace_bytes", "cascade_attn_decode_static",
     "cascade_kernel_timing_begin", "cascade_kernel_timing_end", "cascade_rope_table", "cascade_attn_sharded_rope",
     "cascade_cdelta_shard_map", "cascade_msplit_shard_map", "cascade_index_set_gaps", "cascade_kl_gaps",
-    "cascade_attn_sharded_host",
+    "cascade_attn_sharded_host", "cascade_plan_advance",
 ]
 
 
@@ -83,6 +83,7 @@ def lib() -> ctypes.CDLL:
         L.cascade_index_set_gaps.argtypes = [i32, vp, pi32, pi32, pi32, pi32]
         L.cascade_kl_gaps.argtypes = [i32, vp, vp, i32, vp]
         L.cascade_attn_sharded_host.argtypes = [vp, i32, i32, i32, i32, i32, f32, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.cascade_plan_advance.argtypes = [vp, i32, vp]
         L.cascade_kernel_timing_begin.argtypes = []
         L.cascade_kernel_timing_end.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
         for name in EXPORTS:
@@ -173,6 +174,11 @@ class Plan:
         code = ctypes.c_int32()
         _check(lib().cascade_plan_device_status(self.handle, ctypes.byref(code)))
         return code.value
+
+    def advance(self, q_pos_offset: int):
+        """Move the query block to position ``q_pos_offset`` (token-sharded KV caching): the causal prefixes are
+        recomputed, on the device in the order of the current stream.  A host-only plan needs no stream."""
+        _check(lib().cascade_plan_advance(self.handle, int(q_pos_offset), _stream() if torch.cuda.is_available() else None))
 
     def destroy(self):
         if self.handle:

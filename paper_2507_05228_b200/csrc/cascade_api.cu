@@ -372,6 +372,57 @@ cascade_status_t cascade_plan_dense_mask(const cascade_plan_t* plan, int32_t map
   return CASCADE_OK;
 }
 
+cascade_status_t cascade_plan_advance(cascade_plan_t* plan, int32_t q_pos_offset, void* stream) {
+  if (!plan) {
+    set_error("cascade_plan_advance: null plan");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  const PlanDev& d = plan->dev;
+  const int n_maps = d.n_maps, n_q = d.n_q, n_kv = d.n_kv, J = d.n_q_shards, P = d.n_kv_shards;
+  for (int mp = 0; mp < n_maps; ++mp) {
+    const int32_t* qo = plan->q_off.data() + (size_t)mp * (J + 1);
+    const int32_t* qi = plan->q_idx.data() + (size_t)mp * n_q;
+    const int32_t* ko = plan->kv_off.data() + (size_t)mp * (P + 1);
+    const int32_t* ki = plan->kv_idx.data() + (size_t)mp * n_kv;
+    int32_t* vis = plan->vis.data() + (size_t)mp * n_q * P;
+    for (int k = 0; k < P; ++k) {
+      const int32_t* tb = ki + ko[k];
+      const int32_t* te = ki + ko[k + 1];
+      for (int r = 0; r < n_q; ++r) {
+        int32_t c = (int32_t)(te - tb);  // every key of the shard, unless the mask is causal and cuts the list
+        if (d.causal) {
+          const int64_t pos = (int64_t)qi[r] + q_pos_offset;
+          if (pos < 0) c = 0;
+          else if (pos < n_kv) c = (int32_t)(std::upper_bound(tb, te, (int32_t)pos) - tb);
+        }
+        vis[(size_t)r * P + k] = c;
+      }
+    }
+    uint8_t* pc = plan->pair_class.data() + (size_t)mp * J * P;
+    for (int j = 0; j < J; ++j)
+      for (int k = 0; k < P; ++k) {
+        const int len = ko[k + 1] - ko[k];
+        uint8_t cls = CASCADE_PAIR_EMPTY;
+        if (qo[j + 1] > qo[j] && len > 0) {
+          const int lo = vis[(size_t)qo[j] * P + k], hi = vis[(size_t)(qo[j + 1] - 1) * P + k];
+          cls = hi == 0 ? CASCADE_PAIR_EMPTY : (lo == len ? CASCADE_PAIR_FULL : CASCADE_PAIR_PARTIAL);
+        }
+        pc[(size_t)j * P + k] = cls;
+      }
+  }
+  plan->dev.q_pos_offset = q_pos_offset;
+  if (plan->dev_blob) {
+    // pageable source: the runtime stages it before the call returns, the device copy lands in stream order
+    cudaError_t e = cudaMemcpyAsync(const_cast<int32_t*>(d.vis), plan->vis.data(), plan->vis.size() * 4,
+                                    cudaMemcpyHostToDevice, (cudaStream_t)stream);
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(const_cast<uint8_t*>(d.pair_class), plan->pair_class.data(), plan->pair_class.size(),
+                          cudaMemcpyHostToDevice, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e, "cascade_plan_advance: upload");
+  }
+  return CASCADE_OK;
+}
+
 cascade_status_t cascade_plan_device_status(const cascade_plan_t* plan, int32_t* out_code) {
   if (!plan || !out_code || !plan->dev_blob) {
     set_error("cascade_plan_device_status: null pointer or host-only plan");

@@ -214,3 +214,39 @@ def test_kernel_timing_counts_attention_launches(gu):
     ms2, n2 = cb.cascade_kernel_timing_end()
     assert n2 == 0 and ms2 == 0.0
     plan.destroy()
+
+
+def test_decode_loop_over_a_preallocated_cache_with_plan_advance(gu):
+    """Token-sharded KV caching (Appendix F): one plan over the cache capacity, advanced per generated token.  Rows of
+    the cache beyond the current position hold arbitrary finite values and must not influence the result."""
+    from paper_2507_05228_b200 import binding as cb
+    cap, B, H, Hkv, d, P = 640, 2, 8, 2, 128, 5
+    w = wl.make_workload("cache", B, 1, cap, H, Hkv, d, "bf16", "round_robin", "block_rr", 1, P, seed=41, block=8,
+                         q_pos_offset=0)
+    q, k, v = gu.to_device(w)
+    plan = gu.make_plan(w)
+    steps = [0, 1, 7, 8, 63, 300, 639]
+    for pos in steps:
+        plan.advance(pos)
+        # poison everything the new token must not see
+        k_p, v_p = k.clone(), v.clone()
+        if pos + 1 < cap:
+            k_p[:, pos + 1:] = 3.0e4
+            v_p[:, pos + 1:] = -3.0e4
+        o, lse = cb.cascade_attn_sharded(plan, q, k_p, v_p, w.scale)
+        o_ref, lse_ref = oracle.attention_unsharded(w.q, w.k, w.v, w.scale, causal=True, q_pos_offset=pos)
+        gu.check_output(o, lse, o_ref, lse_ref, w.tol, f"decode at position {pos}")
+        assert int(plan.get("vis")[0].sum()) == pos + 1
+    # a sliding prefill chunk on the tensor-core route
+    w2 = wl.make_workload("chunk_slide", 1, 64, 512, 8, 2, 128, "bf16", "round_robin", "block_rr", 2, 4, seed=42,
+                          block=16, q_pos_offset=0)
+    q, k, v = gu.to_device(w2)
+    plan2 = gu.make_plan(w2)
+    for off in (0, 64, 200, 448):
+        plan2.advance(off)
+        o, lse = cb.cascade_attn_sharded(plan2, q, k, v, w2.scale)
+        o_ref, lse_ref = oracle.attention_unsharded(w2.q, w2.k, w2.v, w2.scale, causal=True, q_pos_offset=off)
+        gu.check_output(o, lse, o_ref, lse_ref, w2.tol, f"prefill chunk at offset {off}")
+    assert plan.device_status() == 0 and plan2.device_status() == 0
+    plan.destroy()
+    plan2.destroy()

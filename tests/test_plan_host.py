@@ -87,3 +87,34 @@ def test_partial_buffer_sizes_match_stage_b_cost_model():
     stat_elems = 2 * beta * N * H
     assert o_elems + stat_elems == beta * (d + 2) * H * N
     assert w.n_kv_shards == beta and w.n_q == N
+
+
+def test_plan_advance_matches_a_plan_built_at_that_position(binding):
+    """Token-sharded KV caching: one plan over the cache capacity, advanced token by token, equals the oracle's plan
+    built for each position (prefix lengths and pair classes bit-exact); the index lists never change."""
+    n_cap, P = 96, 5
+    kv_of = sharding.cdelta_shard_of(n_cap, 4, 20)          # every future slot already has its shard
+    q_of = np.zeros(1, np.int32)
+    plan = binding.cascade_shard_plan_host(q_of, kv_of, 1, P, q_pos_offset=0)
+    kv_idx0 = plan.get("kv_idx").copy()
+    for pos in [0, 1, 3, 4, 19, 20, 57, 95, 96, 200, -1, 7]:
+        plan.advance(pos)
+        ref = oracle.shard_plan(q_of, kv_of, 1, P, q_pos_offset=pos)
+        assert np.array_equal(plan.get("vis")[0], ref.vis), pos
+        assert np.array_equal(plan.get("pair_class")[0], ref.pair_class), pos
+        assert np.array_equal(plan.get("kv_idx"), kv_idx0)
+        assert int(plan.get("vis")[0].sum()) == min(max(pos + 1, 0), n_cap)  # exactly the rows written so far
+    plan.destroy()
+    # a sliding prefill chunk (n_q > 1) and a bidirectional plan (nothing to cut)
+    q_chunk = (np.arange(12) % 3).astype(np.int32)
+    plan = binding.cascade_shard_plan_host(q_chunk, kv_of, 3, P, q_pos_offset=0)
+    for off in (0, 12, 50, 84):
+        plan.advance(off)
+        ref = oracle.shard_plan(q_chunk, kv_of, 3, P, q_pos_offset=off)
+        assert np.array_equal(plan.get("vis")[0], ref.vis) and np.array_equal(plan.get("pair_class")[0], ref.pair_class)
+    plan.destroy()
+    plan = binding.cascade_shard_plan_host(q_chunk, kv_of, 3, P, causal=False)
+    before = plan.get("vis").copy()
+    plan.advance(40)
+    assert np.array_equal(plan.get("vis"), before)
+    plan.destroy()
