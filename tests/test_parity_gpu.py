@@ -78,6 +78,14 @@ def test_non_causal_and_single_shard(gu):
     gu.full_parity(wl.make_workload("one_shard", 1, 300, 300, 4, 2, 128, "bf16", "random", "random", 1, 1, seed=4))
 
 
+def test_non_causal_on_the_tensor_core_route(gu):
+    """Bidirectional mask (the BERT case) in bf16 with head_dim 128: every key of every shard is visible."""
+    gu.full_parity(wl.make_workload("bidir_tc", 2, 384, 384, 8, 2, 128, "bf16", "random", "random", 3, 3, seed=15,
+                                    causal=False))
+    gu.full_parity(wl.make_workload("bidir_tc_cross", 1, 100, 700, 4, 4, 128, "bf16", "round_robin", "block_rr", 2, 5,
+                                    seed=16, causal=False, block=16))
+
+
 def test_chunked_prefill_offsets(gu):
     """n_q < n_kv with the query block at the end of the cache, and a block in the middle."""
     gu.full_parity(wl.make_workload("chunk_end", 2, 96, 400, 8, 2, 128, "bf16", "random", "random", 3, 7, seed=8))
