@@ -48,7 +48,7 @@ struct Vec16<__nv_bfloat16> {
 // statistics (lane `sub` evaluates the weights of parts sub, sub + TPR, ...; weights travel by shuffle) and each lane
 // streams its own 16 bytes of every partial with up to 8 loads in flight.
 template <typename T, int D>
-__global__ void __launch_bounds__(256, 4) merge_kernel(MergeParams p) {
+__global__ void __launch_bounds__(256, 3) merge_kernel(MergeParams p) {
   using VT = Vec16<T>;
   constexpr int V = VT::N;
   constexpr int TPR = D / V;
