@@ -14,7 +14,9 @@
  *  - Pointers named *_dev / q / k / v / o_* / m_* / l_* / workspace are DEVICE pointers owned by the
  *    caller.  Token-to-shard maps and read-back buffers are HOST pointers.
  *  - All GPU work is enqueued on the caller's stream (a cudaStream_t passed as void*; NULL = default
- *    stream) without synchronising, except where a function says it synchronises.
+ *    stream) without synchronising, except where a function says it synchronises.  On the tensor-core route
+ *    the attention grid is launched as a programmatic dependent of the K/V gather grid of the same call, so
+ *    the two overlap; both are ordered after earlier work on the stream and before later work, as usual.
  *  - The library allocates device memory only inside cascade_shard_plan (released by
  *    cascade_plan_destroy).  Scratch memory is caller-provided after cascade_workspace_bytes.
  *  - Token ids, shard ids, rows and positions are 0-based.  Query row i of a sequence sits at position
