@@ -294,7 +294,8 @@ cascade_status_t cascade_kl_gaps(int32_t n_tokens, const uint8_t* r_held, const 
  *                   q, k, v, o and the scratch of one head group.  Overwritten by every call.
  * All work is ordered after what `stream` holds at the time of the call, and `stream` waits for the last output
  * copy: synchronising `stream` makes o_host valid.  The first call on a device creates two internal copy streams and
- * their events (no device memory).  Errors as cascade_attn_sharded, plus CASCADE_ERR_INVALID_ARG for more than 128 KV
+ * their events (no device memory); all calls on a device share them, so calls from several host threads for the same
+ * device must be serialised by the caller.  Errors as cascade_attn_sharded, plus CASCADE_ERR_INVALID_ARG for more than 128 KV
  * heads.
  */
 cascade_status_t cascade_attn_sharded_host(const cascade_plan_t* plan, cascade_dtype_t dtype, int32_t batch,
