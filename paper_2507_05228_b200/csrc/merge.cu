@@ -46,14 +46,16 @@ struct Vec16<__nv_bfloat16> {
 
 // A group of TPR = D / (16 / sizeof(T)) lanes owns one (row, head) output vector.  The lanes share the work on the
 // statistics (lane `sub` evaluates the weights of parts sub, sub + TPR, ...; weights travel by shuffle) and each lane
-// streams its own 16 bytes of every partial with up to 8 loads in flight.
+// streams its own 16 bytes of every partial, two loads in flight per thread at full occupancy (8 CTAs of 256 threads
+// per SM at 32 registers).  Measured on the batched / long prefill partials: 8 loads in flight at 3-4 CTAs per SM
+// 5.4 / 5.9 TB/s, 4 at 6 CTAs 6.0 / 6.4, 2 at 8 CTAs 6.4 / 6.7, 1 at 8 CTAs 5.8 / 6.2.
 template <typename T, int D>
-__global__ void __launch_bounds__(256, 3) merge_kernel(MergeParams p) {
+__global__ void __launch_bounds__(256, 8) merge_kernel(MergeParams p) {
   using VT = Vec16<T>;
   constexpr int V = VT::N;
   constexpr int TPR = D / V;
   constexpr int ITEMS = 256 / TPR;
-  constexpr int CH = TPR < 8 ? TPR : 8;
+  constexpr int CH = 2;  // partial rows in flight per thread
   const int sub = threadIdx.x % TPR;
   const int lane = threadIdx.x & 31;
   const int group_lane0 = lane - sub;
