@@ -3,11 +3,12 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-extras]
 
-One step = one pass of the hot path over one batch of the headline workload (the Llama-8B-shaped prefill
-layer: 2048 tokens, 32 query / 8 KV heads, head_dim 128, bf16, 8 x 8 random shards): the fused call
-``cascade_attn_sharded`` (gather, QK^T, mask, streaming statistics, PV and the post-pass combine in one launch).
-``value`` is algorithmic TFLOP/s = 4 * d * H * (visible query-key pairs) / time, inputs resident in HBM; the
-unfused route (``cascade_attn_partials`` + ``cascade_merge``) and the other workloads are reported next to it.
+One step = one pass of the hot path over one batch of the headline workload, the largest single-GPU prefill
+configuration (the 70B-shaped long-context layer: 32768 tokens, 64 query / 8 KV heads, head_dim 128, bf16, 32 x 32
+random token shards): the fused call ``cascade_attn_sharded`` (shard gather, QK^T, mask, streaming statistics, PV and
+the post-pass combine).  ``value`` is algorithmic TFLOP/s = 4 * d * H * (visible query-key pairs) / time with the
+inputs resident in HBM; the unfused route (``cascade_attn_partials`` + ``cascade_merge``), the other prefill
+configurations, the decode step and the merge are reported next to it, each with its own roofline record.
 Prints ONE JSON line on rank 0.
 """
 from __future__ import annotations
@@ -27,12 +28,28 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 METRIC = "sharded-attn TFLOP/s (prefill)"
-HEADLINE = "c2_prefill_8b"
+HEADLINE = "c4_long_70b"
+HEADLINE_TEXT = ("c4_long_70b: batch 1 per GPU, 32768 tokens, 64 q / 8 kv heads, head_dim 128, bf16, 32x32 random token "
+                 "shards, causal")
 L2_FLUSH_BYTES = 256 << 20
+MIN_STEPS = 20  # timed launches behind every record
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures summarised
-# under profiles/ (None until a capture exists for that workload).
-NCU_TRAFFIC_BYTES = {"c2_prefill_8b": 25463552}  # profiles/attn_tc_kernel_c2_headline.md
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of each record's dominant kernel, from one ncu capture per
+# kernel and workload ((bytes of the captured case, launches of the captured size that make one full-size launch); None =
+# no capture of the kernel as it stands).  The prefill kernel's traffic grows with batch * KV heads (each (sequence, KV
+# head) streams its own K/V and writes its own output rows), the decode and merge kernels' with the batch.
+NCU_TRAFFIC = {
+    "c2_prefill_8b/attn_tc_kernel": None,
+    "c3_batched/attn_tc_kernel": None,
+    "c4_long_70b/attn_tc_kernel": None,
+    "c5_decode/decode_kernel": None,
+    "c3_batched/merge_kernel": None,
+}
+
+
+def _traffic(key):
+    rec = NCU_TRAFFIC.get(key)
+    return None if rec is None else rec[0] * rec[1]
 
 
 def _peaks():
@@ -73,7 +90,7 @@ class ClockSampler:
             self.proc.kill()
         self.tmp.flush()
         self.tmp.seek(0)
-        sm, smax, reasons = [], [], set()
+        sm, smax, power, reasons = [], [], [], set()
         for line in self.tmp.read().splitlines():
             parts = [x.strip() for x in line.split(",")]
             if len(parts) < 9:
@@ -81,6 +98,7 @@ class ClockSampler:
             try:
                 sm.append(float(parts[1]))
                 smax.append(float(parts[2]))
+                power.append(float(parts[3]))
             except ValueError:
                 continue
             for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
@@ -90,7 +108,8 @@ class ClockSampler:
         self.tmp.close()
         os.unlink(self.tmp.name)
         if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm))
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm),
+                       sm_mhz_min=min(sm), power_w_max=max(power))
         return out
 
 
@@ -134,6 +153,204 @@ def _steps_then_kernel(torch, cb, fn, steps, warmup, flush):
     return ms, k_ms / max(k_n, 1), k_n
 
 
+def _tensor_roofline(peaks, kernel, flops, kernel_ms, steps, traffic):
+    achieved = flops / (kernel_ms * 1e-3) / 1e12
+    # a launch of tens of microseconds runs at burst clocks; one of many milliseconds under the power cap
+    return {"bound": "tensor", "kernel": kernel, "achieved": achieved, "peak": peaks["bf16_tflops"],
+            "peak_source": peaks["source"] + " burst bf16 (cuBLAS)", "unit": "TFLOP/s",
+            "frac": achieved / peaks["bf16_tflops"], "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+            "frac_of_nominal_2250": achieved / 2250.0, "kernel_ms": kernel_ms, "steps": steps, "traffic": traffic}
+
+
+def _hbm_roofline(peaks, kernel, nbytes, kernel_ms, steps, traffic):
+    achieved = nbytes / (kernel_ms * 1e-3) / 1e9
+    return {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peaks["hbm_gbs"],
+            "peak_source": peaks["source"] + " copy bandwidth", "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+            "frac_of_8tbs": achieved / 8000.0, "kernel_ms": kernel_ms, "steps": steps, "traffic": traffic,
+            "algorithmic_bytes": nbytes}
+
+
+def plan_statistics(plan, w):
+    """Host-side counts from the plan: how much tensor work the tiling executes per unit of causal work, and the
+    EMPTY / PARTIAL / FULL classes of the (query shard, KV shard) pairs (what pair-class skipping can use)."""
+    vis = plan.get("vis")[0].astype(np.int64)  # [n_q, P]
+    q_off = plan.get("q_off")[0]
+    G = w.H // w.Hkv
+    gp = 1
+    while gp < 8 and G % (2 * gp) == 0:
+        gp *= 2
+    rows_per_cta = 2 * (128 // gp)  # two sub-tiles of 128 MMA rows, gp heads stacked per slot
+    executed = 0
+    for j in range(w.n_q_shards):
+        for r0 in range(q_off[j], q_off[j + 1], rows_per_cta):
+            n = min(rows_per_cta, q_off[j + 1] - r0)
+            need = vis[r0 + n - 1]  # the tile's last row has the longest prefix of every shard
+            keys = int((-(-need // 32) * 32).sum())  # every shard's prefix rounded up to 32-key chunks
+            n_sub = 2 if n > rows_per_cta // 2 else 1
+            executed += keys * n_sub * (128 // gp)  # MMA rows are (slot, head) pairs: 128 / gp slots per sub-tile
+    causal = int(vis.sum())
+    pc = plan.get("pair_class")[0]
+    return {"mma_pairs_executed_over_causal": executed / max(causal, 1),
+            "pair_classes": {"empty": int((pc == 0).sum()), "partial": int((pc == 1).sum()), "full": int((pc == 2).sum())}}
+
+
+ROPE_BASE = 500000.0  # rotary base of the model family the prefill shapes are taken from
+
+
+def measure_prefill(torch, cb, wl, name, flush, peaks, steps, warmup, seed=None, with_rope=True):
+    """Every route of one prefill workload.  Returns (record, context) where context keeps the device tensors alive
+    for callers that go on with the same workload."""
+    w = wl.config(name) if seed is None else wl.config(name, seed=seed)
+    q, k, v = _upload(w, torch, wl)
+    plan = cb.cascade_shard_plan(w.q_shard_of, w.kv_shard_of, w.n_q_shards, w.n_kv_shards, w.q_pos_offset, w.causal)
+    o = torch.empty_like(q)
+    ws = torch.empty(cb.cascade_workspace_bytes(plan, cb.CALL_SHARDED, cb.BF16, w.B, w.H, w.Hkv, w.d),
+                     dtype=torch.uint8, device="cuda")  # shard-major K/V copies, allocated once
+    flops = w.flops()
+
+    def step_fused():
+        cb.cascade_attn_sharded(plan, q, k, v, w.scale, out=o, want_lse=False, workspace=ws)
+
+    launches0 = cb.cascade_launch_count()
+    ms, k_ms, k_n = _steps_then_kernel(torch, cb, step_fused, steps, warmup, flush)
+    launches_per_step = (cb.cascade_launch_count() - launches0) // (2 * steps + warmup + 1)
+    med = statistics.median(ms)
+    rec = {"fused": {"ms": med, "ms_min": min(ms), "tflops": flops / (med * 1e-3) / 1e12, "steps": steps,
+                     "launches_per_step": int(launches_per_step),
+                     "roofline": _tensor_roofline(peaks, "attn_tc_kernel (fused route)", flops, k_ms, k_n,
+                                                  _traffic(name + "/attn_tc_kernel"))}}
+    if with_rope:
+        table = cb.cascade_rope_table(max(w.q_pos_offset + w.n_q, w.n_kv), w.d, ROPE_BASE)
+        ms_r, k_ms_r, _ = _steps_then_kernel(torch, cb, lambda: cb.cascade_attn_sharded_rope(
+            plan, q, k, v, w.scale, table, out=o, want_lse=False, workspace=ws), MIN_STEPS, 3, flush)
+        med_r = statistics.median(ms_r)
+        rec["fused_rope"] = {"ms": med_r, "attn_kernel_ms": k_ms_r, "extra_ms": med_r - med, "steps": MIN_STEPS,
+                             "separate_rotary_pass_bytes":
+                                 2 * (w.B * w.n_q * w.H + w.B * w.n_kv * w.Hkv) * w.d * 2}
+        del table
+    # unfused route: the attention-pass of every pair (tensor-bound, plus the partial writes), then the post-pass (HBM)
+    parts = cb.cascade_attn_partials(plan, q, k, v, w.scale, workspace=ws)
+    ms_p, kp_ms, kp_n = _steps_then_kernel(torch, cb, lambda: cb.cascade_attn_partials(
+        plan, q, k, v, w.scale, out=parts, workspace=ws), MIN_STEPS, 2, flush)
+    ms_m = _time_steps(torch, lambda: cb.cascade_merge(*parts, plan.dev_ptr("q_idx"), out=o, want_lse=False), MIN_STEPS,
+                       3, flush)
+    rows = w.B * w.n_q * w.H
+    part_bytes = w.n_kv_shards * rows * (w.d * 2 + 8)
+    merge_bytes = part_bytes + rows * w.d * 2
+    med_p, med_m = statistics.median(ms_p), statistics.median(ms_m)
+    rec["partials"] = {"ms": med_p, "tflops": flops / (med_p * 1e-3) / 1e12, "steps": MIN_STEPS,
+                       "partial_write_gbs": part_bytes / (kp_ms * 1e-3) / 1e9,
+                       "roofline": _tensor_roofline(peaks, "attn_tc_kernel (one launch over all shard pairs)", flops,
+                                                    kp_ms, kp_n, None)}
+    rec["merge"] = {"ms": med_m, "steps": MIN_STEPS,
+                    "roofline": _hbm_roofline(peaks, "merge_kernel", merge_bytes, med_m, MIN_STEPS,
+                                              _traffic(name + "/merge_kernel"))}
+    rec["partials_plus_merge_ms"] = med_p + med_m
+    rec["plan"] = plan_statistics(plan, w)
+    rec["device_status"] = plan.device_status()
+    del parts
+    return rec, (w, plan, q, k, v, o, ws, ms)
+
+
+def measure_decode(torch, cb, wl, flush, peaks):
+    w = wl.config("c5_decode")
+    q, k, v = _upload(w, torch, wl)
+    plan = cb.cascade_shard_plan(w.q_shard_of, w.kv_shard_of, w.n_q_shards, w.n_kv_shards, w.q_pos_offset, w.causal)
+    parts = cb.cascade_attn_partials(plan, q, k, v, w.scale)
+    steps = 2 * MIN_STEPS
+    ms_d, k_ms, k_n = _steps_then_kernel(torch, cb, lambda: cb.cascade_attn_partials(plan, q, k, v, w.scale, out=parts),
+                                         steps, 3, flush)
+    o = torch.empty_like(q)
+    ws = torch.empty(cb.cascade_workspace_bytes(plan, cb.CALL_SHARDED, cb.BF16, w.B, w.H, w.Hkv, w.d),
+                     dtype=torch.uint8, device="cuda")
+    ms_f = _time_steps(torch, lambda: cb.cascade_attn_sharded(plan, q, k, v, w.scale, out=o, want_lse=False,
+                                                             workspace=ws), steps, 3, flush)
+    # a decode-loop step as a serving loop runs it: advance the plan to the new token's position, then decode + merge
+    pos = [w.n_kv - 1]
+
+    def step_loop():
+        plan.advance(pos[0])
+        cb.cascade_attn_sharded(plan, q, k, v, w.scale, out=o, want_lse=False, workspace=ws)
+
+    ms_l = _time_steps(torch, step_loop, steps, 3, flush)
+    rows = w.B * w.n_kv_shards * w.H
+    merge_bytes = rows * (w.d * 2 + 8) + w.B * w.H * w.d * 2
+    med_f = statistics.median(ms_f)
+    rec = {"partials_ms": statistics.median(ms_d), "decode_plus_merge_ms": med_f,
+           "decode_plus_merge_kv_gbs": w.kv_bytes() / (med_f * 1e-3) / 1e9,
+           "decode_step_with_plan_advance_ms": statistics.median(ms_l), "steps": steps,
+           "merge_bytes": merge_bytes, "device_status": plan.device_status(),
+           "roofline": _hbm_roofline(peaks, "decode_kernel<4>", w.kv_bytes(), k_ms, k_n,
+                                     _traffic("c5_decode/decode_kernel"))}
+    plan.destroy()
+    return rec
+
+
+def measure_small_cases(torch, cb, wl, flush):
+    """The shape of the paper's own latency tables, and the host cost of moving a prefill chunk along a cache."""
+    out = {}
+    # one BERT-Base layer's attention, 128-token prompt, bidirectional mask, fp32, (c, delta) = (8, 16) sharding over
+    # alpha = 2 nodes (launch-latency-bound at this size)
+    r_of, alpha = cb.cascade_cdelta_shard_map(128, 8, 16)
+    w = wl.make_workload("bert_base_n128", 1, 128, 128, 12, 12, 64, "f32", "round_robin", "round_robin", alpha, alpha,
+                         seed=5, causal=False)
+    q, k, v = _upload(w, torch, wl)
+    plan = cb.cascade_shard_plan(r_of, r_of, alpha, alpha, 0, False)
+    o = torch.empty_like(q)
+    ms_b = _time_steps(torch, lambda: cb.cascade_attn_sharded(plan, q, k, v, w.scale, out=o, want_lse=False),
+                       MIN_STEPS, 3, flush)
+    parts = cb.cascade_attn_partials(plan, q, k, v, w.scale)
+    ms_bp = _time_steps(torch, lambda: (cb.cascade_attn_partials(plan, q, k, v, w.scale, out=parts),
+                                        cb.cascade_merge(*parts, plan.dev_ptr("q_idx"), out=o, want_lse=False)),
+                        MIN_STEPS, 3, flush)
+    out["bert_base_n128_noncausal_f32"] = {"fused_ms": statistics.median(ms_b),
+                                           "partials_plus_merge_ms": statistics.median(ms_bp), "steps": MIN_STEPS,
+                                           "sharding": "(c, delta) = (8, 16), alpha = 2"}
+    plan.destroy()
+    # chunked prefill over a preallocated cache: a 512-row query block moved along 8192 cache rows, 16 KV shards
+    w = wl.config("c3_batched", B=1, n_q=512, H=8, Hkv=2, outlier_frac=0.0, q_pos_offset=0)
+    plan = cb.cascade_shard_plan(w.q_shard_of, w.kv_shard_of, w.n_q_shards, w.n_kv_shards, 0, True)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    n_adv = 0
+    for off in range(0, w.n_kv - w.n_q + 1, w.n_q):
+        plan.advance(off)
+        n_adv += 1
+    torch.cuda.synchronize()
+    out["plan_advance_sliding_chunk"] = {"host_ms_per_advance": (time.perf_counter() - t0) * 1e3 / n_adv,
+                                         "chunk_rows": w.n_q, "cache_rows": w.n_kv, "kv_shards": w.n_kv_shards}
+    plan.destroy()
+    return out
+
+
+def measure_exchange(torch, cb, cd, wl, flush, rank, world):
+    """The multi-rank form of the path: resident K/V per rank, partials, stage-B all-to-all, local post-pass, on one
+    sequence of the 8B-shaped prefill shape.  With one rank the all-to-all is a local copy (no wire)."""
+    from paper_2507_05228_b200 import exchange as ex
+    w = wl.config("c2_prefill_8b", n_q=8192, n_kv=8192, n_q_shards=16, n_kv_shards=16, seed=11)  # same on every rank
+    q, k, v = _upload(w, torch, wl)
+    ra = ex.RankAttention(w.q_shard_of, w.kv_shard_of, w.n_q_shards, w.n_kv_shards, rank, world)
+    tok = torch.from_numpy(ra.tokens.astype(np.int64)).cuda()
+    k_res, v_res = k[:, tok].contiguous(), v[:, tok].contiguous()
+    del k, v
+    sent = [0]
+
+    def step():
+        _, _, sent[0] = ra.run(q, k_res, v_res, w.scale)
+
+    ms = _time_steps(torch, step, MIN_STEPS, 3, flush)
+    total_ms = cd.max_over_ranks(sum(ms)) / MIN_STEPS
+    wire = cd.sum_over_ranks(float(sent[0]))
+    rec = {"workload": "one 8B-shaped sequence of 8192 tokens, 16 x 16 random shards, KV shards dealt round-robin to "
+                       "the ranks", "world": world, "ms_per_layer": total_ms, "steps": MIN_STEPS,
+           "tflops": w.flops() / (total_ms * 1e-3) / 1e12, "stage_b_bytes_sent": wire,
+           "stage_b_bytes_closed_form": ex.stage_b_bytes(w.B, w.n_kv_shards, w.n_q, w.H, w.d, 2),
+           "wire": "nccl all_to_all_single" if world > 1 else "none (one rank: local copy)",
+           "device_status": ra.plan.device_status()}
+    ra.destroy()
+    return rec
+
+
 def run_ours(args):
     import torch
     from paper_2507_05228_b200 import binding as cb
@@ -149,28 +366,16 @@ def run_ours(args):
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
 
     # ---- headline workload; with N ranks every rank runs its own sequence (independent problems, no exchange)
-    w = wl.config(HEADLINE, seed=1 + rank)
+    w = wl.config(HEADLINE, seed=3 + rank)
     q, k, v = _upload(w, torch, wl)
     plan = cb.cascade_shard_plan(w.q_shard_of, w.kv_shard_of, w.n_q_shards, w.n_kv_shards, w.q_pos_offset, w.causal)
     o = torch.empty_like(q)
-    lse = None
     flops = w.flops()
-
     ws = torch.empty(cb.cascade_workspace_bytes(plan, cb.CALL_SHARDED, cb.BF16, w.B, w.H, w.Hkv, w.d),
-                     dtype=torch.uint8, device="cuda")  # shard-major K/V copies, allocated once
+                     dtype=torch.uint8, device="cuda")
 
     def step_fused():
         cb.cascade_attn_sharded(plan, q, k, v, w.scale, out=o, want_lse=False, workspace=ws)
-
-    parts = None
-
-    def step_unfused():
-        nonlocal parts
-        parts = cb.cascade_attn_partials(plan, q, k, v, w.scale, out=parts, workspace=ws)
-        cb.cascade_merge(*parts, plan.dev_ptr("q_idx"), out=o, want_lse=False)
-
-    step_unfused()  # allocate the partial buffers once
-    torch.cuda.synchronize()
 
     sampler = ClockSampler(local) if rank == 0 else None
     cd.barrier()
@@ -182,18 +387,25 @@ def run_ours(args):
     cd.barrier()
     wall = time.perf_counter() - wall0
     launches = (cb.cascade_launch_count() - launches0) * args.steps // (args.steps + args.warmup)
-    # the same steps once more with the library's event pairs around every launch of the attention kernel
+    # Two launches per step: the shard gather of K/V (HBM-bound, tens of microseconds) and the attention kernel, which
+    # dominates.  Its own duration comes from the event pairs the library records around it in a second pass of the
+    # same steps, under the same clock sampling: in the timed steps the two launches overlap (programmatic dependent
+    # launch), and an event between them would take that overlap away.
     _time_steps(torch, step_fused, args.steps, 1, flush, after_warmup=cb.cascade_kernel_timing_begin)
     kernel_ms_total, kernel_launches = cb.cascade_kernel_timing_end()
     clocks = sampler.stop() if sampler else None
     total_ms = cd.max_over_ranks(sum(ms))
     ms_per_step = total_ms / args.steps
     value = world * flops / (ms_per_step * 1e-3) / 1e12
+    kernel_ms = kernel_ms_total / max(kernel_launches, 1)
+    roofline = _tensor_roofline(peaks, "attn_tc_kernel (fused route)", flops, kernel_ms, kernel_launches,
+                                _traffic(HEADLINE + "/attn_tc_kernel"))
+    roofline["timed"] = "second pass of the same steps, event pair around each attention launch"
+    status = plan.device_status()
 
     # ---- end to end through the public call with host buffers: H2D of q, k, v, the fused call, D2H of o
     hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
     ho = torch.empty_like(hq).pin_memory()
-
     ws_host = torch.empty(cb.cascade_workspace_bytes(plan, cb.CALL_SHARDED_HOST, cb.BF16, w.B, w.H, w.Hkv, w.d),
                           dtype=torch.uint8, device="cuda")
 
@@ -202,63 +414,54 @@ def run_ours(args):
         # one KV head group after another with the copies in both directions and the compute overlapped
         cb.cascade_attn_sharded_host(plan, hq, hk, hv, w.scale, ho, ws_host)
 
-    e2e_steps = max(3, min(args.steps, 50))
+    e2e_steps = max(3, min(args.steps, 10))
     ms_e2e = _time_steps(torch, step_e2e, e2e_steps, 3, flush)
     e2e_ms = cd.max_over_ranks(sum(ms_e2e)) / e2e_steps
     h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv))
     d2h = ho.numel() * ho.element_size()
-
-    ms_unfused = _time_steps(torch, step_unfused, max(3, min(args.steps, 50)), 3, flush)
-    status = plan.device_status()
-    routes = {
-        "fused": {"ms": statistics.median(ms), "ms_min": min(ms), "tflops": flops / (statistics.median(ms) * 1e-3) / 1e12},
-        "partials_merge": {"ms": statistics.median(ms_unfused), "ms_min": min(ms_unfused),
-                           "tflops": flops / (statistics.median(ms_unfused) * 1e-3) / 1e12},
-    }
-    # Two launches per step: the shard gather of K/V (HBM-bound, a few microseconds) and the attention kernel, which
-    # dominates.  Its own duration comes from the event pairs the library recorded around it in a second pass of the
-    # same steps, under the same clock sampling: in the timed steps the two launches overlap (programmatic dependent
-    # launch), and an event between them would take that overlap away.
-    kernel_ms = kernel_ms_total / max(kernel_launches, 1)
-    achieved = flops / (kernel_ms * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": "attn_tc_kernel (fused route)", "achieved": achieved,
-                "peak": peaks["bf16_tflops"], "peak_source": peaks["source"] + " burst bf16 (cuBLAS)",
-                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
-                "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"], "frac_of_nominal_2250": achieved / 2250.0,
-                "kernel_ms": kernel_ms, "kernel_launches_timed": kernel_launches,
-                "timed": "second pass of the same steps, event pair around each attention launch",
-                "traffic": NCU_TRAFFIC_BYTES.get(HEADLINE)}
-    if rank == 0 and world == 1 and not args.no_extras:
-        routes["fused_rope"] = _rope_record(torch, cb, w, plan, q, k, v, o, ws, flush, routes["fused"]["ms"], kernel_ms,
-                                            steps=max(args.steps, 20))
+    del hq, hk, hv, ho, ws_host
+    plan_stats = plan_statistics(plan, w)
     plan.destroy()
-    del q, k, v, o, parts
+    del q, k, v, o, ws
+    torch.cuda.empty_cache()
 
-    extras = {}
+    exchange = None
+    if not args.no_extras:
+        exchange = measure_exchange(torch, cb, cd, wl, flush, rank, world)
+
+    workloads = {}
     if rank == 0 and world == 1 and not args.no_extras:
-        extras = run_extras(torch, cb, wl, flush, peaks)
+        for name, steps in (("c4_long_70b", MIN_STEPS), ("c3_batched", 2 * MIN_STEPS), ("c2_prefill_8b", 10 * MIN_STEPS)):
+            rec, ctx = measure_prefill(torch, cb, wl, name, flush, peaks, steps, 3)
+            ctx[1].destroy()
+            del ctx
+            torch.cuda.empty_cache()
+            workloads[name] = rec
+        workloads["c5_decode"] = measure_decode(torch, cb, wl, flush, peaks)
+        workloads.update(measure_small_cases(torch, cb, wl, flush))
 
     cpu = None
     if rank == 0 and world == 1:
-        cpu = cpu_baseline(wl.config(HEADLINE, seed=1))
+        cpu = cpu_baseline(w)  # rank 0's own sequence: the arrays the GPU steps ran on
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": HEADLINE + ": batch 1 per GPU, 2048 tokens, 32 q / 8 kv heads, head_dim 128, "
-                                              "8x8 random token shards, causal", "route": "cascade_attn_sharded (fused)",
-                       "l2": "flushed between steps (256 MiB write)", "sequences_per_gpu": 1},
+            "config": {"workload": HEADLINE_TEXT, "route": "cascade_attn_sharded (fused)",
+                       "l2": "flushed between steps (256 MiB write); inputs are 1.2 GB", "sequences_per_gpu": 1,
+                       "plan": plan_stats},
             "clocks": clocks,
             "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
-                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "call": "cascade_attn_sharded_host (pinned host buffers; copies and compute pipelined over KV heads)"},
             "gpu_launches": int(launches),
             "roofline": roofline,
             "cpu_baseline": cpu,
-            "routes": routes,
-            "other_workloads": extras,
+            "ms_median": statistics.median(ms), "ms_min": min(ms),
+            "exchange": exchange,
+            "other_workloads": workloads,
             "device_status": status,
             "wall_s_timed_region": wall,
         }
@@ -266,129 +469,37 @@ def run_ours(args):
     cd.finalize()
 
 
-ROPE_BASE = 500000.0  # rotary base of the model family the prefill shapes are taken from
+def _oracle_rows(w, n_rows):
+    """Evenly spaced query rows (token ids) of the workload, the last row included."""
+    return np.unique(np.linspace(0, w.n_q - 1, max(2, n_rows)).astype(np.int32))
 
 
-def _rope_record(torch, cb, w, plan, q, k, v, o, ws, flush, plain_ms, plain_kernel_ms, steps=5):
-    """The fused route with the rotary step of the pre-pass folded into the staging of Q and K rows: what the extra
-    arithmetic costs over the same call on rotated inputs (a separate rotary pass would read and write Q and K once)."""
-    table = cb.cascade_rope_table(max(w.q_pos_offset + w.n_q, w.n_kv), w.d, ROPE_BASE)
-    ms, k_ms, k_n = _steps_then_kernel(torch, cb, lambda: cb.cascade_attn_sharded_rope(
-        plan, q, k, v, w.scale, table, out=o, want_lse=False, workspace=ws), steps, 3, flush)
-    med = statistics.median(ms)
-    qk_bytes = 2 * (w.B * w.n_q * w.H + w.B * w.n_kv * w.Hkv) * w.d * 2  # one read + one write of Q and K
-    return {"rope_fused_ms": med, "rope_attn_kernel_ms": k_ms, "rope_extra_ms": med - plain_ms,
-            "rope_attn_kernel_extra_ms": k_ms - plain_kernel_ms,
-            "separate_rotary_pass_bytes": qk_bytes}
-
-
-def run_extras(torch, cb, wl, flush, peaks):
-    """The other prefill workloads (tensor-bound) and the decode step and merge (HBM-bound), a few steps each."""
-    out = {}
-    for name in ("c3_batched", "c4_long_70b"):
-        w = wl.config(name)
-        q, k, v = _upload(w, torch, wl)
-        plan = cb.cascade_shard_plan(w.q_shard_of, w.kv_shard_of, w.n_q_shards, w.n_kv_shards, w.q_pos_offset, w.causal)
-        o = torch.empty_like(q)
-        ws = torch.empty(cb.cascade_workspace_bytes(plan, cb.CALL_SHARDED, cb.BF16, w.B, w.H, w.Hkv, w.d),
-                         dtype=torch.uint8, device="cuda")
-        ms, k_ms, k_n = _steps_then_kernel(torch, cb, lambda: cb.cascade_attn_sharded(
-            plan, q, k, v, w.scale, out=o, want_lse=False, workspace=ws), 5, 3, flush)
-        tf = w.flops() / (statistics.median(ms) * 1e-3) / 1e12
-        ktf = w.flops() / (k_ms * 1e-3) / 1e12  # attention kernel alone (without the K/V shard gather)
-        rec = {"fused_ms": statistics.median(ms), "fused_tflops": tf, "frac_of_burst_peak": tf / peaks["bf16_tflops"],
-               "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"], "frac_of_nominal_2250": tf / 2250.0,
-               "attn_kernel_ms": k_ms, "attn_kernel_tflops": ktf,
-               "attn_kernel_frac_of_burst_peak": ktf / peaks["bf16_tflops"]}
-        rec.update(_rope_record(torch, cb, w, plan, q, k, v, o, ws, flush, rec["fused_ms"], rec["attn_kernel_ms"]))
-        # unfused route: partials (tensor) then merge (HBM)
-        parts = cb.cascade_attn_partials(plan, q, k, v, w.scale, workspace=ws)
-        ms_p = _time_steps(torch, lambda: cb.cascade_attn_partials(plan, q, k, v, w.scale, out=parts, workspace=ws), 3, 2,
-                           flush)
-        ms_m = _time_steps(torch, lambda: cb.cascade_merge(*parts, plan.dev_ptr("q_idx"), out=o, want_lse=False), 5, 3,
-                           flush)
-        rows = w.B * w.n_q * w.H
-        merge_bytes = w.n_kv_shards * rows * (w.d * 2 + 8) + rows * w.d * 2
-        gbs = merge_bytes / (statistics.median(ms_m) * 1e-3) / 1e9
-        rec.update(partials_ms=statistics.median(ms_p),
-                   partials_tflops=w.flops() / (statistics.median(ms_p) * 1e-3) / 1e12,
-                   merge_ms=statistics.median(ms_m), merge_gbs=gbs, merge_frac_of_hbm=gbs / peaks["hbm_gbs"],
-                   merge_frac_of_8tbs=gbs / 8000.0)
-        out[name] = rec
-        plan.destroy()
-        del q, k, v, o, parts, ws
-        torch.cuda.empty_cache()
-    w = wl.config("c5_decode")
-    q, k, v = _upload(w, torch, wl)
-    plan = cb.cascade_shard_plan(w.q_shard_of, w.kv_shard_of, w.n_q_shards, w.n_kv_shards, w.q_pos_offset, w.causal)
-    parts = cb.cascade_attn_partials(plan, q, k, v, w.scale)
-    ms_d = _time_steps(torch, lambda: cb.cascade_attn_partials(plan, q, k, v, w.scale, out=parts), 20, 3, flush)
-    o = torch.empty_like(q)
-    nbytes = cb.cascade_workspace_bytes(plan, cb.CALL_SHARDED, cb.BF16, w.B, w.H, w.Hkv, w.d)
-    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
-    ms_f = _time_steps(torch, lambda: cb.cascade_attn_sharded(plan, q, k, v, w.scale, out=o, want_lse=False,
-                                                             workspace=ws), 20, 3, flush)
-    # a decode-loop step as a serving loop runs it: advance the plan to the new token's position, then decode + merge
-    pos = [w.n_kv - 1]
-
-    def step_loop():
-        plan.advance(pos[0])
-        cb.cascade_attn_sharded(plan, q, k, v, w.scale, out=o, want_lse=False, workspace=ws)
-
-    ms_l = _time_steps(torch, step_loop, 20, 3, flush)
-    gbs = w.kv_bytes() / (statistics.median(ms_d) * 1e-3) / 1e9
-    out["c5_decode"] = {"decode_step_with_plan_advance_ms": statistics.median(ms_l),
-                        "partials_ms": statistics.median(ms_d), "kv_gbs": gbs, "frac_of_hbm": gbs / peaks["hbm_gbs"],
-                        "frac_of_8tbs": gbs / 8000.0, "decode_plus_merge_ms": statistics.median(ms_f),
-                        "decode_plus_merge_kv_gbs": w.kv_bytes() / (statistics.median(ms_f) * 1e-3) / 1e9}
-    plan.destroy()
-    del q, k, v, o, parts, ws
-    # The shape of the paper's own latency tables: one BERT-Base layer's attention, 128-token prompt, bidirectional
-    # mask, fp32, (c, delta) = (8, 16) sharding over alpha = 2 nodes (launch-latency-bound at this size).
-    r_of, alpha = cb.cascade_cdelta_shard_map(128, 8, 16)
-    w = wl.make_workload("bert_base_n128", 1, 128, 128, 12, 12, 64, "f32", "round_robin", "round_robin", alpha, alpha,
-                         seed=5, causal=False)
-    q, k, v = _upload(w, torch, wl)
-    plan = cb.cascade_shard_plan(r_of, r_of, alpha, alpha, 0, False)
-    o = torch.empty_like(q)
-    ms_b = _time_steps(torch, lambda: cb.cascade_attn_sharded(plan, q, k, v, w.scale, out=o, want_lse=False), 20, 3,
-                       flush)
-    parts = cb.cascade_attn_partials(plan, q, k, v, w.scale)
-    ms_bp = _time_steps(torch, lambda: (cb.cascade_attn_partials(plan, q, k, v, w.scale, out=parts),
-                                        cb.cascade_merge(*parts, plan.dev_ptr("q_idx"), out=o, want_lse=False)), 20, 3,
-                        flush)
-    out["bert_base_n128_noncausal_f32"] = {"fused_ms": statistics.median(ms_b),
-                                           "partials_plus_merge_ms": statistics.median(ms_bp),
-                                           "sharding": "(c, delta) = (8, 16), alpha = 2"}
-    plan.destroy()
-    return out
+def _pairs(w, rows):
+    return float(np.clip(rows.astype(np.int64) + w.q_pos_offset + 1, 0, w.n_kv).sum()) * w.B
 
 
 def cpu_baseline(w, budget_s: float = 20.0):
-    """The fp64 oracle as it stands, timed on this machine's host cores on a bounded sample of the workload."""
+    """The fp64 oracle as it stands, timed on this machine's host cores on a bounded sample of the workload: evenly
+    spaced query rows (all heads), as many as the budget allows.  `value` is the rate on that sample; the time the
+    whole workload would take at that rate is given as an extrapolation."""
     import oracle
     cores = oracle.num_threads()
-    probe = np.arange(w.n_q - 32, w.n_q, dtype=np.int32)  # 32 of the most expensive rows
+    probe = np.arange(w.n_q - 16, w.n_q, dtype=np.int32)  # 16 of the most expensive rows
     t0 = time.perf_counter()
     oracle.attention_unsharded(w.q, w.k, w.v, w.scale, causal=w.causal, q_pos_offset=w.q_pos_offset, rows=probe)
-    t_probe = time.perf_counter() - t0
-    pairs_probe = float(np.clip(probe + w.q_pos_offset + 1, 0, w.n_kv).sum())
-    rate = pairs_probe / max(t_probe, 1e-6)  # visible pairs per second (all heads)
-    total_pairs = w.visible_pairs() / w.B
-    if total_pairs / rate <= budget_s:
-        rows = np.arange(w.n_q, dtype=np.int32)
-        sample = f"all {w.n_q} query rows of {w.name}, all heads"
-    else:
-        n = max(8, int(w.n_q * budget_s * rate / total_pairs))
-        rows = np.unique(np.linspace(0, w.n_q - 1, n).astype(np.int32))
-        sample = f"{rows.size} evenly spaced query rows of {w.name}, all heads"
+    rate = _pairs(w, probe) / max(time.perf_counter() - t0, 1e-6)  # visible pairs per second (all heads)
+    total_pairs = float(w.visible_pairs())
+    n = int(min(w.n_q, max(8, w.n_q * budget_s * rate / total_pairs)))
+    rows = _oracle_rows(w, n)
     t0 = time.perf_counter()
     oracle.attention_unsharded(w.q, w.k, w.v, w.scale, causal=w.causal, q_pos_offset=w.q_pos_offset, rows=rows)
     dt = time.perf_counter() - t0
-    pairs = float(np.clip(rows.astype(np.int64) + w.q_pos_offset + 1, 0, w.n_kv).sum()) * w.B
+    pairs = _pairs(w, rows)
     fl = 4.0 * w.d * w.H * pairs
+    sample = (f"all {w.n_q} query rows" if rows.size == w.n_q else f"{rows.size} evenly spaced query rows") + \
+             f" of {w.name}, all heads"
     return {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample,
-            "seconds": dt}
+            "seconds": dt, "whole_workload_seconds_extrapolated": dt * total_pairs / pairs}
 
 
 def run_reference(args):
@@ -399,18 +510,16 @@ def run_reference(args):
         return
     import oracle
     from paper_2507_05228_b200 import workloads as wl
-    w = wl.config(HEADLINE, seed=1)
+    w = wl.config(HEADLINE, seed=3)
     cores = oracle.num_threads()
     probe = np.arange(w.n_q - 16, w.n_q, dtype=np.int32)
     t0 = time.perf_counter()
     oracle.attention_unsharded(w.q, w.k, w.v, w.scale, rows=probe)
-    rate = float((probe + 1).sum()) / max(time.perf_counter() - t0, 1e-6)
-    budget = 120.0 / max(1, args.steps + args.warmup)
-    pairs_per_row = (w.n_q + 1) / 2.0
-    n_rows = int(max(4, min(w.n_q, budget * rate / pairs_per_row)))
-    rows = np.unique(np.linspace(0, w.n_q - 1, n_rows).astype(np.int32))
-    pairs = float((rows.astype(np.int64) + 1).sum())
-    fl = 4.0 * w.d * w.H * pairs
+    rate = _pairs(w, probe) / max(time.perf_counter() - t0, 1e-6)
+    budget = 100.0 / max(1, args.steps + args.warmup)
+    n_rows = int(max(4, min(w.n_q, w.n_q * budget * rate / float(w.visible_pairs()))))
+    rows = _oracle_rows(w, n_rows)
+    fl = 4.0 * w.d * w.H * _pairs(w, rows)
     for _ in range(args.warmup):
         oracle.attention_unsharded(w.q, w.k, w.v, w.scale, rows=rows)
     t0 = time.perf_counter()
@@ -423,7 +532,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": HEADLINE + " (fp64 CPU oracle, unsharded definition)", "sample": sample},
+        "config": {"workload": HEADLINE_TEXT, "arm": "fp64 CPU oracle, unsharded definition", "sample": sample},
         "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -433,10 +542,10 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=3000)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=60)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--no-extras", action="store_true", help="skip the other workloads (c3, c4, c5)")
+    ap.add_argument("--no-extras", action="store_true", help="skip the other workloads and routes")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":

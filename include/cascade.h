@@ -4,8 +4,8 @@
  * The paper (Cascade: Token-Sharded Private LLM Inference) splits the tokens of a layer into disjoint
  * index sets -- query shards S_j and key/value shards T_k (Section 5.1) -- lets one "AttnNode" per pair
  * (j, k) compute a partial attention output u with per-row statistics m (row max) and e (sum of
- * exponentials) (Algorithm 3), and combines the partials over k with a log-sum-exp weighted average
- * (Section 5.2.3, Algorithm 4 lines 1-8), which reproduces unsharded softmax attention exactly.
+ * exponentials) (the Attention-Pass algorithm), and combines the partials over k with a log-sum-exp weighted average
+ * (Section 5.2.3, the Post-Pass algorithm), which reproduces unsharded softmax attention exactly.
  * This library runs all parties on one GPU.
  *
  * Conventions
@@ -24,7 +24,7 @@
  *  - Tensors are token-major: element (b, token, head, c) lives at
  *    base + b*strides.batch + token*strides.token + head*strides.head + c   (units: elements, c contiguous).
  *    Row starts must be 16-byte aligned.
- *  - Query head h reads KV head h / (n_heads / n_kv_heads)  ("repeat_kv", Algorithm 3 lines 1-2).
+ *  - Query head h reads KV head h / (n_heads / n_kv_heads)  ("repeat_kv", the Attention-Pass algorithm).
  *  - "Shard-major row order": query rows listed shard 0 first, then shard 1, ..., ascending token id
  *    inside a shard (Section 5.2.2: rows are concatenated in sorted order).  Slot r of that order holds
  *    token Q_IDX[r].
@@ -114,6 +114,28 @@ cascade_status_t cascade_shard_plan(int32_t n_maps, int32_t n_q, int32_t n_kv, c
                                     int32_t q_pos_offset, int32_t causal, void* stream,
                                     cascade_plan_t** out_plan);
 
+/*
+ * cascade_shard_plan_resident -- a plan for a party that holds only SOME of the K/V rows: an AttnNode keeps the k, v
+ * rows of its own KV shards and nothing else (Section 5.2: every AttnNode_{jk} receives k^{T_k}, v^{T_k}; "Caching" in
+ * the appendix on cost optimizations: each node stores the rows of its shard).  The k/v tensors of the attention calls
+ * then have n_kv = (number of resident rows) rows, and row y is the token at ORIGINAL position kv_pos[y]; the causal
+ * mask compares that position with the query position, so VIS[r][k] = #{y in T_k : kv_pos[y] <= q_idx[r] + q_pos_offset}.
+ *   kv_pos   HOST int32 [n_maps][n_kv], non-negative and strictly ascending inside a map (rows kept in token order)
+ * Everything else as cascade_shard_plan (which is this call with kv_pos[y] = y).  The partials of such a plan are the
+ * columns of the full problem's partials that belong to the resident shards; cascade_merge over the union of all
+ * parties' columns gives the exact result (Section 5.2.3).  cascade_attn_sharded_rope refuses these plans (it takes a
+ * key row's position from its index).  Errors as cascade_shard_plan; BAD_MAP also for a kv_pos that is not ascending.
+ */
+cascade_status_t cascade_shard_plan_resident(int32_t n_maps, int32_t n_q, int32_t n_kv, const int32_t* q_shard_of,
+                                             const int32_t* kv_shard_of, const int32_t* kv_pos, int32_t n_q_shards,
+                                             int32_t n_kv_shards, int32_t q_pos_offset, int32_t causal, void* stream,
+                                             cascade_plan_t** out_plan);
+/* The same, built on the host only (see cascade_shard_plan_host). */
+cascade_status_t cascade_shard_plan_resident_host(int32_t n_maps, int32_t n_q, int32_t n_kv, const int32_t* q_shard_of,
+                                                  const int32_t* kv_shard_of, const int32_t* kv_pos,
+                                                  int32_t n_q_shards, int32_t n_kv_shards, int32_t q_pos_offset,
+                                                  int32_t causal, cascade_plan_t** out_plan);
+
 /* Same arrays as cascade_shard_plan, built on the host only: no CUDA call is made, so it works on a machine
  * without a GPU.  The plan can be read with cascade_plan_get / cascade_plan_dense_mask (device pointers are
  * NULL) and must be destroyed as usual; the attention calls reject it with INVALID_ARG. */
@@ -135,11 +157,16 @@ cascade_status_t cascade_plan_dense_mask(const cascade_plan_t* plan, int32_t map
                                          uint8_t* host_out, int64_t capacity);
 
 /* Reads the plan's device status word (SYNCHRONISES the device): 0 = no kernel that used this plan hit a
- * bounded-wait limit; otherwise a code identifying the wait.  Returns TIMEOUT if non-zero. */
+ * bounded-wait limit; otherwise a code identifying the wait.  Returns TIMEOUT if non-zero.
+ * The word is sticky: once a wait inside the tensor-core kernel has given up (2 s without progress), every later
+ * attention call on this plan returns CASCADE_OK from the host but its blocks exit at once and write nothing.  A
+ * non-zero status therefore invalidates the outputs of every call made on the plan since the last check that read 0;
+ * destroy the plan and build a new one.  A caller that cannot afford stale outputs polls this after the calls whose
+ * results it is about to use. */
 cascade_status_t cascade_plan_device_status(const cascade_plan_t* plan, int32_t* out_code);
 
 /*
- * cascade_attn_partials -- the attention-pass of every AttnNode_{jk} (Algorithm 3) in one launch:
+ * cascade_attn_partials -- the attention-pass of every AttnNode_{jk} (the Attention-Pass algorithm) in one launch:
  * for each query shard j and KV shard k, a = scale * q^{S_j} (k^{T_k})^T + s^{S_j T_k}; m = row max;
  * l = row sum exp(a - m); u = softmax(a) v^{T_k}.  Rows of Q/K/V are gathered through the plan's maps.
  *   q  [batch][n_q][n_heads][head_dim], k, v [batch][n_kv][n_kv_heads][head_dim]  (strides given)
@@ -149,6 +176,10 @@ cascade_status_t cascade_plan_device_status(const cascade_plan_t* plan, int32_t*
  * per sequence, Appendix D.)  batch must equal n_maps when the plan has per-sequence maps.
  * head_dim in {64,128}; bf16 with head_dim 128 runs on the tensor cores (tcgen05), everything else on
  * the fp32 ALU kernel; n_q == 1 with bf16 runs the KV-streaming decode kernel.
+ * scale must be positive and finite (INVALID_ARG otherwise: the kernels take row maxima before scaling).
+ * Only the k/v rows that some query row of the plan sees have to hold finite values: positions later than the last
+ * query position (the unwritten tail of a preallocated cache) may hold anything, NaN bit patterns included; no route
+ * lets them reach a result.  batch and n_heads may not exceed 65535 (and batch * n_kv_shards on the ALU route).
  * workspace: as reported by cascade_workspace_bytes(CASCADE_CALL_PARTIALS) (may be 0 -> NULL allowed).  The
  * tensor-core route first copies K and V into shard-major order there (the stage-A hand-over of each KV shard to
  * its AttnNodes, Appendix D): 2 * batch * n_kv_heads * n_kv * head_dim * 2 bytes, overwritten by every call.
@@ -162,7 +193,7 @@ cascade_status_t cascade_attn_partials(const cascade_plan_t* plan, cascade_dtype
                                        void* stream);
 
 /*
- * cascade_merge -- the post-pass combine (Algorithm 4 lines 1-8; derivation in Section 5.2.3):
+ * cascade_merge -- the post-pass combine (the Post-Pass algorithm; derivation in Section 5.2.3):
  * n = max_p m_p;  w = sum_p exp(m_p - n) l_p;  o = sum_p exp(m_p - n) l_p u_p / w.
  * Needs no plan.  Inputs in the layout cascade_attn_partials writes, with n_parts = n_kv_shards.
  *   row_scatter  DEVICE int32 [n_rows] or NULL: output token row of partial row r (the plan's Q_IDX
@@ -179,8 +210,7 @@ cascade_status_t cascade_merge(cascade_dtype_t dtype, int32_t batch, int32_t n_p
                                float* lse_out, void* stream);
 
 /*
- * cascade_attn_sharded -- attention-pass and post-pass fused (Algorithm 3 followed by Algorithm 4 lines
- * 1-8): walks the KV shards of the plan one after another for each query-shard tile and carries
+ * cascade_attn_sharded -- attention-pass and post-pass fused (the Attention-Pass algorithm followed by the Post-Pass algorithm): walks the KV shards of the plan one after another for each query-shard tile and carries
  * (n, w, o) across shards, so no partial is written to memory; by the identity of Section 5.2.3 the
  * result equals cascade_merge(cascade_attn_partials(...)).  Output in token order:
  *   o_out [batch][n_q][n_heads][head_dim] with strides; lse_out optional fp32 [batch][n_q][n_heads].
@@ -197,8 +227,8 @@ cascade_status_t cascade_attn_sharded(const cascade_plan_t* plan, cascade_dtype_
                                       size_t workspace_bytes, void* stream);
 
 /*
- * cascade_rope_table -- the positional table p of the rotary embedding (Section 4 lists p among the tensors set up
- * before inference and sharded with the tokens; Algorithm 2 consumes its rows p^{R_i}).  The paper does not print
+ * cascade_rope_table -- the positional table p of the rotary embedding (Section 5.1 lists p among the tensors set up
+ * before inference and sharded with the tokens; the Pre-Pass algorithm consumes its rows p^{R_i}).  The paper does not print
  * the rotary formula; this library takes the rotate-half form with theta_i = base^(-2 i / head_dim):
  *   table[t][i] = (cos(t theta_i), sin(t theta_i)),  t = 0 .. n_positions-1,  i = 0 .. head_dim/2 - 1,
  * angles formed and evaluated in fp64, stored as fp32 pairs.
@@ -210,7 +240,7 @@ cascade_status_t cascade_rope_table(int32_t n_positions, int32_t head_dim, doubl
                                     void* stream);
 
 /*
- * cascade_attn_sharded_rope -- cascade_attn_sharded with the tail of the pre-pass fused in (Algorithm 2:
+ * cascade_attn_sharded_rope -- cascade_attn_sharded with the tail of the pre-pass fused in (the Pre-Pass algorithm:
  * q <- rotary_pos_emb(q, p^{R_i}), k <- rotary_pos_emb(k, p^{R_i})): q and k are given UNROTATED; every query row is
  * turned by the table row of its position (q_pos_offset + token index) and every key row by the row of its token
  * index while they are staged for the attention kernel, so no separate pass over q and k runs:
@@ -314,6 +344,8 @@ cascade_status_t cascade_attn_sharded_host(const cascade_plan_t* plan, cascade_d
  * stream order); the index lists do not change.  Works for any n_q (a prefill chunk that slides along the sequence);
  * the work-sorted order of the plan's query tiles is left as it was built, which affects speed only.
  * Calls that use the plan before and after must be on `stream` or ordered with it.
+ * Cache rows beyond the new position need not be initialised (see cascade_attn_partials); rows at or before it must be
+ * written, and finite, before the attention call that follows.
  * Errors: CASCADE_ERR_INVALID_ARG (null plan), CASCADE_ERR_CUDA.
  */
 cascade_status_t cascade_plan_advance(cascade_plan_t* plan, int32_t q_pos_offset, void* stream);

@@ -128,7 +128,7 @@ def dense_mask(plan: Plan, j: int, k: int) -> np.ndarray:
 
 
 def attn_pass(q, k, v, scale, plan: Plan, row_tokens=None):
-    """Per-(query shard, KV shard) partials, Algorithm 3.  Returns (u, m, e) in fp64 with
+    """Per-(query shard, KV shard) partials, the Attention-Pass algorithm.  Returns (u, m, e) in fp64 with
     u [B, n_kv_shards, n_rows, H, d] and m, e [B, n_kv_shards, n_rows, H]; rows are the query tokens listed in
     ``row_tokens`` (default: every slot in shard-major order, plan.q_idx)."""
     lib = _load()
@@ -154,7 +154,7 @@ def attn_pass(q, k, v, scale, plan: Plan, row_tokens=None):
 
 
 def post_pass(u, m, e, row_scatter=None):
-    """Log-sum-exp combine over parts, Algorithm 4 lines 1-8.  Returns (o [B,n_rows,H,d], lse)."""
+    """Log-sum-exp combine over parts, the Post-Pass algorithm.  Returns (o [B,n_rows,H,d], lse)."""
     lib = _load()
     u = np.ascontiguousarray(u, np.float64)
     m = np.ascontiguousarray(m, np.float64)

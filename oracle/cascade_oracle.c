@@ -40,8 +40,8 @@ int oracle_num_threads(void) {
 #endif
 }
 
-/* KV head serving query head h: the paper broadcasts H_KV heads to H ("repeat_kv", Algorithm 3
- * lines 1-2); contiguous groups of G = H / H_KV query heads share one KV head. */
+/* KV head serving query head h: the paper broadcasts H_KV heads to H ("repeat_kv" in the Attention-Pass
+ * algorithm); contiguous groups of G = H / H_KV query heads share one KV head. */
 static inline int kv_head_of(int h, int H, int Hkv) { return h / (H / Hkv); }
 
 /* scale * <q_row, k_row> in double */
@@ -179,15 +179,16 @@ int oracle_shard_plan(int n_q, int n_kv, const int32_t* q_shard_of, const int32_
 }
 
 /*
- * Attention-pass of every AttnNode_{jk} (Algorithm 3), one (query shard, KV shard) pair at a time,
- * step by step as printed:   a = scale * q k^T + s ;  m = row_max(a) ;  a = exp(a - m) ;
- * e = row_sum(a) ;  a = a / e ;  u = a v.
- * The mask s is 0 where KV position <= query position and -inf elsewhere (all 0 if !causal).
+ * Attention-pass of every AttnNode_{jk} (the AttnNode Single Layer Attention-Pass algorithm; the derived tensors m,
+ * e, u of Section 5.1), from their definitions, one (query row, head, KV shard) at a time:
+ *   a_y = scale * q . k_y  for the keys y of T_kk that the row may see (KV position <= query position; all of T_kk
+ *         if !causal) -- the sharded mask s^{S_j T_kk} removes the others;
+ *   m   = max_y a_y,   e = sum_y exp(a_y - m),   u = (sum_y exp(a_y - m) v_y) / e.
  * Rows evaluated: the n_rows query tokens listed in row_tok (normally q_idx, i.e. every slot in shard-major
  * order; a subset is allowed so that large cases can be sampled).  Outputs:
  *   u[B][n_kv_shards][n_rows][H][d],  m,e[B][n_kv_shards][n_rows][H]   (double).
- * A row that sees no key of the shard has m = -inf, e = 0, u = 0 (the printed steps would divide by
- * zero there; the post-pass gives such a term weight zero).
+ * A row that sees no key of the shard has m = -inf, e = 0, u = 0 (the definitions would divide by zero there; the
+ * post-pass gives such a term weight zero).
  */
 void oracle_attn_pass(int B, int n_q, int n_kv, int H, int Hkv, int d, double scale,
                       int q_pos_offset, int causal, const float* q, const float* k, const float* v,
@@ -197,6 +198,7 @@ void oracle_attn_pass(int B, int n_q, int n_kv, int H, int Hkv, int d, double sc
 #pragma omp parallel
   {
     double* a = (double*)malloc(sizeof(double) * (size_t)(n_kv > 0 ? n_kv : 1));
+    int32_t* seen = (int32_t*)malloc(sizeof(int32_t) * (size_t)(n_kv > 0 ? n_kv : 1));
 #pragma omp for schedule(dynamic, 16)
     for (long job = 0; job < total; ++job) {
       const int h = (int)(job % H);
@@ -207,47 +209,48 @@ void oracle_attn_pass(int B, int n_q, int n_kv, int H, int Hkv, int d, double sc
       const int tok = row_tok[r];
       const long pos = (long)tok + q_pos_offset;
       const float* qr = q + (((size_t)b * n_q + tok) * H + h) * d;
-      const int lo = kv_off[kk], hi = kv_off[kk + 1], len = hi - lo;
       const size_t stat = (((size_t)b * n_kv_shards + kk) * n_rows + r) * H + h;
       double* urow = u + stat * d;
       for (int c = 0; c < d; ++c) urow[c] = 0.0;
-      /* line 3: masked logits of this row against the whole shard */
+      /* the keys of T_kk this row may see, and their scaled logits */
+      int n_seen = 0;
       double mx = -INFINITY;
-      for (int s2 = 0; s2 < len; ++s2) {
-        const int y = kv_idx[lo + s2];
-        const double mask = (!causal || (long)y <= pos) ? 0.0 : -INFINITY;
-        a[s2] = logit(qr, k + (((size_t)b * n_kv + y) * Hkv + g) * d, d, scale) + mask;
-        if (a[s2] > mx) mx = a[s2]; /* line 4 */
+      for (int s2 = kv_off[kk]; s2 < kv_off[kk + 1]; ++s2) {
+        const int y = kv_idx[s2];
+        if (causal && (long)y > pos) continue;
+        seen[n_seen] = y;
+        a[n_seen] = logit(qr, k + (((size_t)b * n_kv + y) * Hkv + g) * d, d, scale);
+        if (a[n_seen] > mx) mx = a[n_seen];
+        ++n_seen;
       }
-      if (len == 0 || mx == -INFINITY) {
+      if (n_seen == 0) {
         m[stat] = -INFINITY;
         e[stat] = 0.0;
         continue;
       }
       double sum = 0.0;
-      for (int s2 = 0; s2 < len; ++s2) {
-        a[s2] = exp(a[s2] - mx); /* line 5 */
-        sum += a[s2];            /* line 6 */
+      for (int t = 0; t < n_seen; ++t) {
+        const double w = exp(a[t] - mx);
+        sum += w;
+        const float* vr = v + (((size_t)b * n_kv + seen[t]) * Hkv + g) * d;
+        for (int c = 0; c < d; ++c) urow[c] += w * (double)vr[c];
       }
-      for (int s2 = 0; s2 < len; ++s2) {
-        const double w = a[s2] / sum; /* line 7 */
-        if (w == 0.0) continue;
-        const float* vr = v + (((size_t)b * n_kv + kv_idx[lo + s2]) * Hkv + g) * d;
-        for (int c = 0; c < d; ++c) urow[c] += w * (double)vr[c]; /* line 8 */
-      }
+      for (int c = 0; c < d; ++c) urow[c] /= sum;
       m[stat] = mx;
       e[stat] = sum;
     }
     free(a);
+    free(seen);
   }
 }
 
 /*
- * Post-pass combine (Algorithm 4 lines 1-8), for every row and head:
- *   n = max_k m_k ;  w = sum_k exp(m_k - n) e_k ;  o = sum_k exp(m_k - n) e_k u_k / w.
+ * Post-pass combine (the CompNode Single Layer Post-Pass algorithm up to the attention output; identity of
+ * Section 5.2.3), for every row and head over the parts p:
+ *   n = max_p m_p ;  w = sum_p exp(m_p - n) e_p ;  o = (sum_p exp(m_p - n) e_p u_p) / w.
  * Inputs in the layout oracle_attn_pass writes (parts = KV shards).  Output rows go back to token
  * order when row_scatter (= q_idx) is given: o[B][n_rows][H][d], lse[B][n_rows][H] = n + log w.
- * Terms with e_k = 0 (m_k = -inf) contribute nothing; if all terms are empty o = 0, lse = -inf.
+ * Parts with e_p = 0 (m_p = -inf) contribute nothing; if all parts are empty o = 0, lse = -inf.
  */
 void oracle_post_pass(int B, int n_parts, int n_rows, int H, int d, const double* u, const double* m,
                       const double* e, const int32_t* row_scatter, double* o, double* lse) {
@@ -259,9 +262,8 @@ void oracle_post_pass(int B, int n_parts, int n_rows, int H, int d, const double
     const int b = (int)(job / ((long)H * n_rows));
     const int out_row = row_scatter ? row_scatter[r] : r;
     double* orow = o + (((size_t)b * n_rows + out_row) * H + h) * d;
-    for (int c = 0; c < d; ++c) orow[c] = 0.0; /* line 1 */
-    double w = 0.0;                            /* line 2 */
-    double nmax = -INFINITY;                   /* line 3 */
+    for (int c = 0; c < d; ++c) orow[c] = 0.0;
+    double nmax = -INFINITY;
     for (int p = 0; p < n_parts; ++p) {
       const double mp = m[(((size_t)b * n_parts + p) * n_rows + r) * H + h];
       if (mp > nmax) nmax = mp;
@@ -270,15 +272,16 @@ void oracle_post_pass(int B, int n_parts, int n_rows, int H, int d, const double
       lse[((size_t)b * n_rows + out_row) * H + h] = -INFINITY;
       continue;
     }
-    for (int p = 0; p < n_parts; ++p) { /* line 4 */
+    double w = 0.0;
+    for (int p = 0; p < n_parts; ++p) {
       const size_t stat = (((size_t)b * n_parts + p) * n_rows + r) * H + h;
       if (e[stat] == 0.0) continue;
       const double wt = exp(m[stat] - nmax) * e[stat];
-      w += wt; /* line 5 */
+      w += wt;
       const double* urow = u + stat * d;
-      for (int c = 0; c < d; ++c) orow[c] += wt * urow[c]; /* line 6 */
+      for (int c = 0; c < d; ++c) orow[c] += wt * urow[c];
     }
-    for (int c = 0; c < d; ++c) orow[c] /= w; /* line 8 */
+    for (int c = 0; c < d; ++c) orow[c] /= w;
     lse[((size_t)b * n_rows + out_row) * H + h] = nmax + log(w);
   }
 }

@@ -1,7 +1,7 @@
 """Oracle for the rotary step of the pre-pass -- TEST INFRASTRUCTURE ONLY (numpy, fp64).
 
-Algorithm 2 (CompNode single-layer pre-pass) ends with q <- rotary_pos_emb(q, p^{R_i}) and the same for k,
-where p^{R_i} are the rows of the positional table p (Section 4, notation) at the node's ORIGINAL token
+the Pre-Pass algorithm (CompNode single-layer pre-pass) ends with q <- rotary_pos_emb(q, p^{R_i}) and the same for k,
+where p^{R_i} are the rows of the positional table p (Section 5.1, Sharding and Notation) at the node's ORIGINAL token
 indices R_i.  The paper does not print the rotary formula; the reading taken here is the common
 "rotate-half" form with exact real-valued angles:
 
@@ -21,7 +21,7 @@ import numpy as np
 
 
 def positional_table(n_positions: int, d: int, base: float):
-    """(cos, sin), each float64 [n_positions, d/2]: row t is p[t] (Section 4: p is initialised before inference)."""
+    """(cos, sin), each float64 [n_positions, d/2]: row t is p[t] (Section 5.1: p is initialised before inference)."""
     if d % 2:
         raise ValueError("head_dim must be even")
     i = np.arange(d // 2, dtype=np.float64)
@@ -49,7 +49,7 @@ def round_to_io(x: np.ndarray, dtype: str) -> np.ndarray:
 
 
 def rotary_pos_emb(x: np.ndarray, positions: np.ndarray, base: float, io_dtype: str = "f64") -> np.ndarray:
-    """Algorithm 2, last two steps.  x: [B, n, heads, d]; positions: [n] original token indices of the rows.
+    """the rotary steps of the Pre-Pass algorithm.  x: [B, n, heads, d]; positions: [n] original token indices of the rows.
     Returns float64 holding values rounded to ``io_dtype``."""
     x = np.asarray(x, dtype=np.float64)
     B, n, H, d = x.shape

@@ -30,7 +30,8 @@ EXPORTS = [
     "cascade_merge", "cascade_attn_sharded", "cascade_workspace_bytes", "cascade_attn_decode_static",
     "cascade_kernel_timing_begin", "cascade_kernel_timing_end", "cascade_rope_table", "cascade_attn_sharded_rope",
     "cascade_cdelta_shard_map", "cascade_msplit_shard_map", "cascade_index_set_gaps", "cascade_kl_gaps",
-    "cascade_attn_sharded_host", "cascade_plan_advance",
+    "cascade_attn_sharded_host", "cascade_plan_advance", "cascade_shard_plan_resident",
+    "cascade_shard_plan_resident_host",
 ]
 
 
@@ -62,6 +63,8 @@ def lib() -> ctypes.CDLL:
         L.cascade_launch_count.restype = i64
         L.cascade_shard_plan.argtypes = [i32, i32, i32, vp, vp, i32, i32, i32, i32, vp, ctypes.POINTER(vp)]
         L.cascade_shard_plan_host.argtypes = [i32, i32, i32, vp, vp, i32, i32, i32, i32, ctypes.POINTER(vp)]
+        L.cascade_shard_plan_resident.argtypes = [i32, i32, i32, vp, vp, vp, i32, i32, i32, i32, vp, ctypes.POINTER(vp)]
+        L.cascade_shard_plan_resident_host.argtypes = [i32, i32, i32, vp, vp, vp, i32, i32, i32, i32, ctypes.POINTER(vp)]
         L.cascade_plan_destroy.argtypes = [vp]
         L.cascade_plan_get.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(i64)]
         L.cascade_plan_dense_mask.argtypes = [vp, i32, i32, i32, vp, i64]
@@ -224,6 +227,24 @@ def cascade_shard_plan_host(q_shard_of, kv_shard_of, n_q_shards: int, n_kv_shard
     _check(lib().cascade_shard_plan_host(n_maps, n_q, n_kv, qs.ctypes.data_as(ctypes.c_void_p),
                                          ks.ctypes.data_as(ctypes.c_void_p), n_q_shards, n_kv_shards, q_pos_offset,
                                          int(bool(causal)), ctypes.byref(out)))
+    return Plan(out.value, n_maps, n_q, n_kv, n_q_shards, n_kv_shards)
+
+
+def cascade_shard_plan_resident(q_shard_of, kv_shard_of, kv_pos, n_q_shards: int, n_kv_shards: int,
+                                q_pos_offset: int = 0, causal: bool = True, host_only: bool = False) -> Plan:
+    """Plan for a party that holds only some K/V rows: row y of its k/v tensors is the token at original position
+    kv_pos[y] (int32, strictly ascending; shaped like kv_shard_of)."""
+    qs, ks = _maps(q_shard_of, kv_shard_of)
+    kp = np.ascontiguousarray(np.asarray(kv_pos, dtype=np.int32).reshape(ks.shape))
+    n_maps, n_q = qs.shape
+    n_kv = ks.shape[1]
+    out = ctypes.c_void_p()
+    args = (n_maps, n_q, n_kv, qs.ctypes.data_as(ctypes.c_void_p), ks.ctypes.data_as(ctypes.c_void_p),
+            kp.ctypes.data_as(ctypes.c_void_p), n_q_shards, n_kv_shards, q_pos_offset, int(bool(causal)))
+    if host_only:
+        _check(lib().cascade_shard_plan_resident_host(*args, ctypes.byref(out)))
+    else:
+        _check(lib().cascade_shard_plan_resident(*args, _stream(), ctypes.byref(out)))
     return Plan(out.value, n_maps, n_q, n_kv, n_q_shards, n_kv_shards)
 
 

@@ -1,4 +1,4 @@
-// Attention-pass on the fp32 ALUs (Algorithm 3), used for fp32 inputs and for shapes the tensor-core kernel
+// Attention-pass on the fp32 ALUs (the Attention-Pass algorithm), used for fp32 inputs and for shapes the tensor-core kernel
 // does not take.  One CTA owns a tile of up to 32 query slots of one shard and one head; KV rows of a shard are
 // gathered through the plan's index list into shared memory 32 at a time; each warp owns 8 query rows, one
 // lane per key for the logits and one lane per output column group for the value product.  Statistics follow
@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(128) attn_simt_kernel(AttnParams p) {
         const int r = warp * RPW + rr;
         const int my_vis = sVis[r];
         if (t0 >= my_vis) continue;  // warp-uniform: nothing of this tile is visible to the row
-        // line 3: logits, lane = key
+        // logits a = scale q k^T, lane = key
         float dot = 0.f;
 #pragma unroll
         for (int c = 0; c < D; c += 4) {
@@ -139,7 +139,7 @@ __global__ void __launch_bounds__(128) attn_simt_kernel(AttnParams p) {
       }
     }
     if (!p.fused) {
-      // write the pair's (u, m, l): u normalised inside the shard (Algorithm 3 line 7)
+      // write the pair's (u, m, l): u normalised inside the shard (the Attention-Pass algorithm)
 #pragma unroll
       for (int rr = 0; rr < RPW; ++rr) {
         const int r = warp * RPW + rr;

@@ -1,13 +1,13 @@
 // Attention-pass on the 5th-generation tensor cores (tcgen05 + TMEM) for bf16, head_dim 128.
 //
 // Work decomposition.  The M dimension of one MMA tile (128 rows) is filled with (query slot, head) pairs: the
-// Gp query heads that read the same KV head ("repeat_kv", Algorithm 3 lines 1-2) are stacked next to each other,
+// Gp query heads that read the same KV head ("repeat_kv", the Attention-Pass algorithm) are stacked next to each other,
 // so a tile covers only 128 / Gp consecutive slots of one query shard.  Under token sharding the rows of a shard
 // are spread over the whole sequence, and the staircase between the shortest and the longest visible prefix of a
 // tile is wasted tensor work; stacking heads shrinks that staircase by Gp.
 // One CTA owns two such sub-tiles (the next 128 / Gp slots of the same shard, same heads), which share every K/V
-// tile, and either one KV shard (partials: Algorithm 3 for the pair) or all KV shards one after another (fused:
-// the carry n, w, o of Algorithm 4 is the running max / sum / output of the streaming softmax).
+// tile, and either one KV shard (partials: the Attention-Pass algorithm for the pair) or all KV shards one after another (fused:
+// the carry n, w, o of the Post-Pass algorithm is the running max / sum / output of the streaming softmax).
 // The KV shards are walked one after another; each shard's visible prefix (as seen by the CTA's last row, which has
 // the longest one) is cut into chunks of 32 keys, and four consecutive chunks of that stream - possibly from
 // different shards - form one MMA tile of 128 keys, so that only the last tile of a CTA is narrower.  (An MMA costs
@@ -311,7 +311,7 @@ struct TmaArgs {
 };
 
 // kRope: the query rows are turned by the rotary embedding of their positions while they are staged (the key rows
-// were turned by the gather pass), Algorithm 2.
+// were turned by the gather pass), the Pre-Pass algorithm.
 template <bool kRope>
 __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_constant__ AttnParams p, int lg,
                                                               int tile_major,
@@ -603,7 +603,8 @@ if constexpr (kRope) {
             mx[q4] = fmax3(mx[q4], __uint_as_float(sr[32 * q4 + j]), __uint_as_float(sr[32 * q4 + j + 1]));
           mx[q4] = fmaxf(mx[q4], __uint_as_float(sr[32 * q4 + 31]));
         }
-        const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c;
+        const float smax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));  // raw logit
+        const float tmax = smax * c;
         m_true = fmaxf(m_true, tmax);
         float m_new = m_run;
         if (m_run == -INFINITY || m_true > m_run + kRescaleThreshold) m_new = m_true;
@@ -642,7 +643,14 @@ if constexpr (kRope) {
         }
         float psum0, psum1;
         unpack2(psum2, psum0, psum1);
-        l_run = l_run * alpha + (psum0 + psum1);
+        // The tensor core multiplies the weights after rounding them to bf16, while the sum above is taken before.
+        // With the lagging reference max even the largest weight of a row has an arbitrary mantissa, so when one key
+        // dominates a row its rounding error (up to 2^-9 relative) would go straight into O / l: 0.009 at |v| = 4.5.
+        // The sum therefore takes the tile's largest weight as the tensor core sees it (same fma and ex2 as in the
+        // loop above, so the same bits); the other weights' errors are small against l or average out.
+        const float p_top = ex2(fmaf(smax, c, neg_m));
+        const float p_top_seen = __uint_as_float(pack_bf16x2(0.f, p_top) & 0xffff0000u);
+        l_run = l_run * alpha + ((psum0 + psum1) + (p_top_seen - p_top));
         // S_FULL(i) was committed after PV(i-1), so the output accumulator is quiescent until this thread's
         // arrival on P_FULL(i) below
         if (i > 0 && __any_sync(0xffffffffu, changed)) {
@@ -889,6 +897,19 @@ bool encode_sorted(CUtensorMap* map, const void* base, int64_t n_kv, int64_t n_m
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Number of SMs of the current device (queried once per device).
+int sm_count() {
+  static int cached[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
 }  // namespace
 
 cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void* v_sorted, cudaStream_t stream) {
@@ -907,7 +928,7 @@ cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void
   const int n_parts = p.fused ? 1 : p.plan.n_kv_shards;
   const int64_t n_ctas = (int64_t)p.plan.n_qtiles[3 - lg] * (p.H >> lg) * p.batch * n_parts;
   if (n_ctas >= (int64_t)1 << 31) return cudaErrorInvalidConfiguration;
-  const int tile_major = n_ctas <= 8 * 148;  // few CTAs per SM: balance matters more than L2 locality
+  const int tile_major = n_ctas <= 8 * (int64_t)sm_count();  // few CTAs per SM: balance matters more than L2 locality
   TimedLaunch timed(stream);
   // Programmatic dependent launch on the gather grid that precedes it in the stream: the set-up of the CTAs overlaps
   // the gather's tail.  Not while kernel timing is recording: the event between the two launches must separate them.

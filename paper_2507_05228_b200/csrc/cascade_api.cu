@@ -4,6 +4,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <cmath>
 #include <atomic>
 #include <new>
 
@@ -80,13 +81,60 @@ static void build_qtiles(const cascade_plan& pl, int map, int rows_per_tile, std
   for (auto& t : tiles) out.push_back(t.t);
 }
 
+// Visible-prefix lengths vis[r][k] of one map: the number of keys of shard k (a list of K/V rows, ascending) whose
+// position is <= the position of query slot r.  A K/V row sits at position kv_pos[row] (its own index if kv_pos is null).
+static void fill_vis(const cascade_plan& pl, int mp, int q_pos_offset, int32_t* vis) {
+  const PlanDev& d = pl.dev;
+  const int n_q = d.n_q, n_kv = d.n_kv, P = d.n_kv_shards;
+  const int32_t* qi = pl.q_idx.data() + (size_t)mp * n_q;
+  const int32_t* ko = pl.kv_off.data() + (size_t)mp * (P + 1);
+  const int32_t* ki = pl.kv_idx.data() + (size_t)mp * n_kv;
+  const int32_t* kp = pl.kv_pos.empty() ? nullptr : pl.kv_pos.data() + (size_t)mp * n_kv;
+  for (int k = 0; k < P; ++k) {
+    const int32_t* tb = ki + ko[k];
+    const int32_t* te = ki + ko[k + 1];
+    for (int r = 0; r < n_q; ++r) {
+      int32_t c = (int32_t)(te - tb);  // every key of the shard, unless the mask is causal and cuts the list
+      if (d.causal) {
+        const int64_t pos = (int64_t)qi[r] + q_pos_offset;
+        if (kp) {
+          c = (int32_t)(std::upper_bound(tb, te, pos, [kp](int64_t x, int32_t row) { return x < kp[row]; }) - tb);
+        } else if (pos < 0) {
+          c = 0;
+        } else if (pos < n_kv) {
+          c = (int32_t)(std::upper_bound(tb, te, (int32_t)pos) - tb);
+        }
+      }
+      vis[(size_t)r * P + k] = c;
+    }
+  }
+}
+
+// EMPTY / PARTIAL / FULL per (query shard, KV shard) from the prefix lengths of the shard's first and last row
+// (rows ascend in position, so the first row has the shortest prefix and the last the longest).
+static void fill_pair_class(const cascade_plan& pl, int mp, const int32_t* vis, uint8_t* pc) {
+  const int J = pl.dev.n_q_shards, P = pl.dev.n_kv_shards;
+  const int32_t* qo = pl.q_off.data() + (size_t)mp * (J + 1);
+  const int32_t* ko = pl.kv_off.data() + (size_t)mp * (P + 1);
+  for (int j = 0; j < J; ++j)
+    for (int k = 0; k < P; ++k) {
+      const int len = ko[k + 1] - ko[k];
+      uint8_t cls = CASCADE_PAIR_EMPTY;
+      if (qo[j + 1] > qo[j] && len > 0) {
+        const int lo = vis[(size_t)qo[j] * P + k], hi = vis[(size_t)(qo[j + 1] - 1) * P + k];
+        cls = hi == 0 ? CASCADE_PAIR_EMPTY : (lo == len ? CASCADE_PAIR_FULL : CASCADE_PAIR_PARTIAL);
+      }
+      pc[(size_t)j * P + k] = cls;
+    }
+}
+
 }  // namespace cascade
 
 using namespace cascade;
 
 extern "C" {
 
-int32_t cascade_version(void) { return 100; }
+int32_t cascade_version(void) { return 101; }
 const char* cascade_last_error(void) { return g_err; }
 int64_t cascade_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
@@ -113,8 +161,9 @@ cascade_status_t cascade_kernel_timing_end(double* total_ms, int64_t* n_launches
 }
 
 static cascade_status_t plan_host(int32_t n_maps, int32_t n_q, int32_t n_kv, const int32_t* q_shard_of,
-                                  const int32_t* kv_shard_of, int32_t n_q_shards, int32_t n_kv_shards,
-                                  int32_t q_pos_offset, int32_t causal, cascade_plan_t** out_plan) {
+                                  const int32_t* kv_shard_of, const int32_t* kv_pos, int32_t n_q_shards,
+                                  int32_t n_kv_shards, int32_t q_pos_offset, int32_t causal,
+                                  cascade_plan_t** out_plan) {
   if (!out_plan || !q_shard_of || !kv_shard_of) {
     set_error("cascade_shard_plan: null pointer");
     return CASCADE_ERR_INVALID_ARG;
@@ -136,6 +185,15 @@ static cascade_status_t plan_host(int32_t n_maps, int32_t n_q, int32_t n_kv, con
                 n_kv_shards);
       return CASCADE_ERR_BAD_MAP;
     }
+  if (kv_pos)
+    for (int mp = 0; mp < n_maps; ++mp)
+      for (int y = 0; y < n_kv; ++y) {
+        const int32_t* kp = kv_pos + (size_t)mp * n_kv;
+        if (kp[y] < 0 || (y > 0 && kp[y] <= kp[y - 1])) {
+          set_error("cascade_shard_plan: kv_pos must be non-negative and strictly ascending (map %d, row %d)", mp, y);
+          return CASCADE_ERR_BAD_MAP;
+        }
+      }
   cascade_plan* pl = new (std::nothrow) cascade_plan();
   if (!pl) {
     set_error("cascade_shard_plan: host allocation failed");
@@ -157,8 +215,10 @@ static cascade_status_t plan_host(int32_t n_maps, int32_t n_q, int32_t n_kv, con
     pl->q_inv.assign((size_t)n_maps * n_q, 0);
     pl->kv_idx.assign((size_t)n_maps * n_kv, 0);
     pl->kv_inv.assign((size_t)n_maps * n_kv, 0);
+    pl->kv_slot_shard.assign((size_t)n_maps * n_kv, 0);
     pl->vis.assign((size_t)n_maps * n_q * P, 0);
     pl->pair_class.assign((size_t)n_maps * J * P, 0);
+    if (kv_pos) pl->kv_pos.assign(kv_pos, kv_pos + (size_t)n_maps * n_kv);
     int max_len = 0;
     // counting sort of token ids by shard id: ascending ids inside every shard
     auto sort_by_shard = [](const int32_t* shard_of, int n, int S, int32_t* off, int32_t* idx, int32_t* inv) {
@@ -179,38 +239,14 @@ static cascade_status_t plan_host(int32_t n_maps, int32_t n_q, int32_t n_kv, con
       int32_t* ki = pl->kv_idx.data() + (size_t)mp * n_kv;
       sort_by_shard(q_shard_of + (size_t)mp * n_q, n_q, J, qo, qi, pl->q_inv.data() + (size_t)mp * n_q);
       sort_by_shard(kv_shard_of + (size_t)mp * n_kv, n_kv, P, ko, ki, pl->kv_inv.data() + (size_t)mp * n_kv);
-      int32_t* vis = pl->vis.data() + (size_t)mp * n_q * P;
+      int32_t* slot_shard = pl->kv_slot_shard.data() + (size_t)mp * n_kv;
       for (int k = 0; k < P; ++k) {
-        const int32_t* tb = ki + ko[k];
-        const int32_t* te = ki + ko[k + 1];
-        max_len = std::max(max_len, (int)(te - tb));
-        for (int r = 0; r < n_q; ++r) {
-          int32_t c;
-          if (!causal) {
-            c = (int32_t)(te - tb);
-          } else {
-            const int64_t pos = (int64_t)qi[r] + q_pos_offset;
-            if (pos < 0) c = 0;
-            else if (pos >= n_kv) c = (int32_t)(te - tb);
-            else c = (int32_t)(std::upper_bound(tb, te, (int32_t)pos) - tb);
-          }
-          vis[(size_t)r * P + k] = c;
-        }
+        max_len = std::max(max_len, (int)(ko[k + 1] - ko[k]));
+        std::fill(slot_shard + ko[k], slot_shard + ko[k + 1], k);
       }
-      uint8_t* pc = pl->pair_class.data() + (size_t)mp * J * P;
-      for (int j = 0; j < J; ++j)
-        for (int k = 0; k < P; ++k) {
-          const int len = ko[k + 1] - ko[k];
-          uint8_t cls = CASCADE_PAIR_EMPTY;
-          if (qo[j + 1] > qo[j] && len > 0) {
-            // rows ascend in position, so the first row has the shortest prefix and the last the longest
-            const int lo = vis[(size_t)qo[j] * P + k], hi = vis[(size_t)(qo[j + 1] - 1) * P + k];
-            if (hi == 0) cls = CASCADE_PAIR_EMPTY;
-            else if (lo == len) cls = CASCADE_PAIR_FULL;
-            else cls = CASCADE_PAIR_PARTIAL;
-          }
-          pc[(size_t)j * P + k] = cls;
-        }
+      int32_t* vis = pl->vis.data() + (size_t)mp * n_q * P;
+      fill_vis(*pl, mp, q_pos_offset, vis);
+      fill_pair_class(*pl, mp, vis, pl->pair_class.data() + (size_t)mp * J * P);
     }
     pl->dev.max_kv_shard_len = max_len;
     // tile lists, padded to the same length for every map
@@ -238,16 +274,28 @@ static cascade_status_t plan_host(int32_t n_maps, int32_t n_q, int32_t n_kv, con
 cascade_status_t cascade_shard_plan_host(int32_t n_maps, int32_t n_q, int32_t n_kv, const int32_t* q_shard_of,
                                          const int32_t* kv_shard_of, int32_t n_q_shards, int32_t n_kv_shards,
                                          int32_t q_pos_offset, int32_t causal, cascade_plan_t** out_plan) {
-  return plan_host(n_maps, n_q, n_kv, q_shard_of, kv_shard_of, n_q_shards, n_kv_shards, q_pos_offset, causal,
+  return plan_host(n_maps, n_q, n_kv, q_shard_of, kv_shard_of, nullptr, n_q_shards, n_kv_shards, q_pos_offset, causal,
                    out_plan);
 }
 
-cascade_status_t cascade_shard_plan(int32_t n_maps, int32_t n_q, int32_t n_kv, const int32_t* q_shard_of,
-                                    const int32_t* kv_shard_of, int32_t n_q_shards, int32_t n_kv_shards,
-                                    int32_t q_pos_offset, int32_t causal, void* stream,
+cascade_status_t cascade_shard_plan_resident_host(int32_t n_maps, int32_t n_q, int32_t n_kv, const int32_t* q_shard_of,
+                                                  const int32_t* kv_shard_of, const int32_t* kv_pos,
+                                                  int32_t n_q_shards, int32_t n_kv_shards, int32_t q_pos_offset,
+                                                  int32_t causal, cascade_plan_t** out_plan) {
+  if (!kv_pos) {
+    set_error("cascade_shard_plan_resident_host: null kv_pos");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  return plan_host(n_maps, n_q, n_kv, q_shard_of, kv_shard_of, kv_pos, n_q_shards, n_kv_shards, q_pos_offset, causal,
+                   out_plan);
+}
+
+static cascade_status_t plan_device(int32_t n_maps, int32_t n_q, int32_t n_kv, const int32_t* q_shard_of,
+                                    const int32_t* kv_shard_of, const int32_t* kv_pos, int32_t n_q_shards,
+                                    int32_t n_kv_shards, int32_t q_pos_offset, int32_t causal, void* stream,
                                     cascade_plan_t** out_plan) {
   cascade_plan* pl = nullptr;
-  cascade_status_t hs = plan_host(n_maps, n_q, n_kv, q_shard_of, kv_shard_of, n_q_shards, n_kv_shards,
+  cascade_status_t hs = plan_host(n_maps, n_q, n_kv, q_shard_of, kv_shard_of, kv_pos, n_q_shards, n_kv_shards,
                                   q_pos_offset, causal, &pl);
   if (hs != CASCADE_OK) return hs;
   *out_plan = nullptr;
@@ -265,6 +313,7 @@ cascade_status_t cascade_shard_plan(int32_t n_maps, int32_t n_q, int32_t n_kv, c
       {pl->vis.data(), pl->vis.size() * 4, 0},           {pl->pair_class.data(), pl->pair_class.size(), 0},
       {pl->qtiles[0].data(), pl->qtiles[0].size() * 16, 0}, {pl->qtiles[1].data(), pl->qtiles[1].size() * 16, 0},
       {pl->qtiles[2].data(), pl->qtiles[2].size() * 16, 0}, {pl->qtiles[3].data(), pl->qtiles[3].size() * 16, 0},
+      {pl->kv_slot_shard.data(), pl->kv_slot_shard.size() * 4, 0},
   };
   static_assert(kNumTileSizes == 4, "one upload segment per tile list");
   size_t total = 256;  // status word first
@@ -300,8 +349,29 @@ cascade_status_t cascade_shard_plan(int32_t n_maps, int32_t n_q, int32_t n_kv, c
   pl->dev.vis = (const int32_t*)(base + segs[6].off);
   pl->dev.pair_class = (const uint8_t*)(base + segs[7].off);
   for (int ts = 0; ts < kNumTileSizes; ++ts) pl->dev.qtiles[ts] = (const int4*)(base + segs[8 + ts].off);
+  pl->dev.kv_slot_shard = (const int32_t*)(base + segs[12].off);
   *out_plan = pl;
   return CASCADE_OK;
+}
+
+cascade_status_t cascade_shard_plan(int32_t n_maps, int32_t n_q, int32_t n_kv, const int32_t* q_shard_of,
+                                    const int32_t* kv_shard_of, int32_t n_q_shards, int32_t n_kv_shards,
+                                    int32_t q_pos_offset, int32_t causal, void* stream,
+                                    cascade_plan_t** out_plan) {
+  return plan_device(n_maps, n_q, n_kv, q_shard_of, kv_shard_of, nullptr, n_q_shards, n_kv_shards, q_pos_offset,
+                     causal, stream, out_plan);
+}
+
+cascade_status_t cascade_shard_plan_resident(int32_t n_maps, int32_t n_q, int32_t n_kv, const int32_t* q_shard_of,
+                                             const int32_t* kv_shard_of, const int32_t* kv_pos, int32_t n_q_shards,
+                                             int32_t n_kv_shards, int32_t q_pos_offset, int32_t causal, void* stream,
+                                             cascade_plan_t** out_plan) {
+  if (!kv_pos) {
+    set_error("cascade_shard_plan_resident: null kv_pos");
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  return plan_device(n_maps, n_q, n_kv, q_shard_of, kv_shard_of, kv_pos, n_q_shards, n_kv_shards, q_pos_offset, causal,
+                     stream, out_plan);
 }
 
 cascade_status_t cascade_plan_destroy(cascade_plan_t* plan) {
@@ -378,37 +448,11 @@ cascade_status_t cascade_plan_advance(cascade_plan_t* plan, int32_t q_pos_offset
     return CASCADE_ERR_INVALID_ARG;
   }
   const PlanDev& d = plan->dev;
-  const int n_maps = d.n_maps, n_q = d.n_q, n_kv = d.n_kv, J = d.n_q_shards, P = d.n_kv_shards;
+  const int n_maps = d.n_maps, n_q = d.n_q, J = d.n_q_shards, P = d.n_kv_shards;
   for (int mp = 0; mp < n_maps; ++mp) {
-    const int32_t* qo = plan->q_off.data() + (size_t)mp * (J + 1);
-    const int32_t* qi = plan->q_idx.data() + (size_t)mp * n_q;
-    const int32_t* ko = plan->kv_off.data() + (size_t)mp * (P + 1);
-    const int32_t* ki = plan->kv_idx.data() + (size_t)mp * n_kv;
     int32_t* vis = plan->vis.data() + (size_t)mp * n_q * P;
-    for (int k = 0; k < P; ++k) {
-      const int32_t* tb = ki + ko[k];
-      const int32_t* te = ki + ko[k + 1];
-      for (int r = 0; r < n_q; ++r) {
-        int32_t c = (int32_t)(te - tb);  // every key of the shard, unless the mask is causal and cuts the list
-        if (d.causal) {
-          const int64_t pos = (int64_t)qi[r] + q_pos_offset;
-          if (pos < 0) c = 0;
-          else if (pos < n_kv) c = (int32_t)(std::upper_bound(tb, te, (int32_t)pos) - tb);
-        }
-        vis[(size_t)r * P + k] = c;
-      }
-    }
-    uint8_t* pc = plan->pair_class.data() + (size_t)mp * J * P;
-    for (int j = 0; j < J; ++j)
-      for (int k = 0; k < P; ++k) {
-        const int len = ko[k + 1] - ko[k];
-        uint8_t cls = CASCADE_PAIR_EMPTY;
-        if (qo[j + 1] > qo[j] && len > 0) {
-          const int lo = vis[(size_t)qo[j] * P + k], hi = vis[(size_t)(qo[j + 1] - 1) * P + k];
-          cls = hi == 0 ? CASCADE_PAIR_EMPTY : (lo == len ? CASCADE_PAIR_FULL : CASCADE_PAIR_PARTIAL);
-        }
-        pc[(size_t)j * P + k] = cls;
-      }
+    fill_vis(*plan, mp, q_pos_offset, vis);
+    fill_pair_class(*plan, mp, vis, plan->pair_class.data() + (size_t)mp * J * P);
   }
   plan->dev.q_pos_offset = q_pos_offset;
   if (plan->dev_blob) {
@@ -456,7 +500,7 @@ static bool strides_ok(const cascade_strides_t& s, size_t es) {
 }
 
 static cascade_status_t check_attn_args(const char* fn, const cascade_plan_t* plan, cascade_dtype_t dtype,
-                                        int32_t batch, int32_t H, int32_t Hkv, int32_t d, const void* q,
+                                        int32_t batch, int32_t H, int32_t Hkv, int32_t d, float scale, const void* q,
                                         const cascade_strides_t& qs, const void* k, const cascade_strides_t& ks,
                                         const void* v, const cascade_strides_t& vs) {
   if (!plan || !q || !k || !v) {
@@ -473,6 +517,11 @@ static cascade_status_t check_attn_args(const char* fn, const cascade_plan_t* pl
   }
   if (batch < 1 || H < 1 || Hkv < 1) {
     set_error("%s: batch and head counts must be positive", fn);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (!(scale > 0.f) || !std::isfinite(scale)) {
+    // the kernels take row maxima of the raw logits and scale afterwards, which needs a positive factor
+    set_error("%s: scale must be positive and finite", fn);
     return CASCADE_ERR_INVALID_ARG;
   }
   if (H % Hkv != 0) {
@@ -493,8 +542,8 @@ static cascade_status_t check_attn_args(const char* fn, const cascade_plan_t* pl
     set_error("%s: q/k/v pointers and row strides must be 16-byte aligned", fn);
     return CASCADE_ERR_INVALID_ARG;
   }
-  if ((int64_t)batch * std::max(plan->dev.n_kv_shards, 1) > 65535) {
-    set_error("%s: batch * n_kv_shards exceeds 65535", fn);
+  if (batch > 65535 || H > 65535) {  // grid dimensions of the gather, decode and ALU kernels
+    set_error("%s: batch and n_heads may not exceed 65535", fn);
     return CASCADE_ERR_UNSUPPORTED;
   }
   return CASCADE_OK;
@@ -637,7 +686,7 @@ cascade_status_t cascade_attn_partials(const cascade_plan_t* plan, cascade_dtype
                                        void* o_part, float* m_part, float* l_part, void* workspace,
                                        size_t workspace_bytes, void* stream) {
   cascade_status_t s = check_attn_args("cascade_attn_partials", plan, dtype, batch, n_heads, n_kv_heads,
-                                       head_dim, q, q_strides, k, k_strides, v, v_strides);
+                                       head_dim, scale, q, q_strides, k, k_strides, v, v_strides);
   if (s != CASCADE_OK) return s;
   if (!o_part || !m_part || !l_part) {
     set_error("cascade_attn_partials: null output pointer");
@@ -661,6 +710,10 @@ cascade_status_t cascade_attn_partials(const cascade_plan_t* plan, cascade_dtype
     cascade_status_t ws = run_tc(p, "cascade_attn_partials", plan, workspace, workspace_bytes, st, &e);
     if (ws != CASCADE_OK) return ws;
   } else {
+    if ((int64_t)batch * plan->dev.n_kv_shards > 65535) {  // grid z of the ALU kernel on this route
+      set_error("cascade_attn_partials: batch * n_kv_shards exceeds 65535 on the route without tensor cores");
+      return CASCADE_ERR_UNSUPPORTED;
+    }
     e = launch_attn_simt(p, dtype, st);
   }
   if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_partials: launch");
@@ -720,7 +773,7 @@ static cascade_status_t attn_sharded_impl(const char* fn, const cascade_plan_t* 
                                           const float* rope_table, int32_t n_positions, void* o_out,
                                           cascade_strides_t o_strides, float* lse_out, void* workspace,
                                           size_t workspace_bytes, void* stream) {
-  cascade_status_t s = check_attn_args(fn, plan, dtype, batch, n_heads, n_kv_heads, head_dim, q, q_strides, k,
+  cascade_status_t s = check_attn_args(fn, plan, dtype, batch, n_heads, n_kv_heads, head_dim, scale, q, q_strides, k,
                                        k_strides, v, v_strides);
   if (s != CASCADE_OK) return s;
   if (!o_out) {
@@ -742,6 +795,11 @@ static cascade_status_t attn_sharded_impl(const char* fn, const cascade_plan_t* 
     if (n_positions < need) {
       set_error("%s: the positional table has %d rows, the plan needs %lld", fn, n_positions, (long long)need);
       return CASCADE_ERR_INVALID_ARG;
+    }
+    if (!plan->kv_pos.empty()) {
+      set_error("%s: the rotary step takes a key row's position from its index, which a plan over resident K/V rows "
+                "(cascade_shard_plan_resident) does not have", fn);
+      return CASCADE_ERR_UNSUPPORTED;
     }
     if (use_decode(plan, dtype, n_heads, n_kv_heads, head_dim) || !use_tc(plan, dtype, head_dim)) {
       set_error("%s: the rotary step is fused on the tensor-core route only (bf16, head_dim 128, more than one query "

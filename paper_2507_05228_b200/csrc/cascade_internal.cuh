@@ -21,6 +21,7 @@ struct PlanDev {
   const int32_t* kv_off;
   const int32_t* kv_idx;
   const int32_t* kv_inv;
+  const int32_t* kv_slot_shard;  // [n_kv]: the shard whose list holds this position of kv_idx
   const int32_t* vis;
   const uint8_t* pair_class;
   // Query tiles that never cross a shard boundary: {first slot, rows, shard, unused}; rows == 0 pads.
@@ -52,7 +53,7 @@ struct AttnParams {
   void* o_out;
   Strides os;
   float* lse_out;
-  // Rotary step of the pre-pass fused into the staging of Q and K rows (Algorithm 2): rows of the positional table,
+  // Rotary step of the pre-pass fused into the staging of Q and K rows (the Pre-Pass algorithm): rows of the positional table,
   // rope[position * 64 + i] = (cos, sin) of position * theta_i; null = rows are used as given.  A query row sits at
   // position q_pos_offset + token, a key row at its token index.
   const float2* rope;
@@ -74,7 +75,8 @@ struct MergeParams {
 
 struct cascade_plan {
   cascade::PlanDev dev;
-  std::vector<int32_t> q_off, q_idx, q_inv, kv_off, kv_idx, kv_inv, vis;
+  std::vector<int32_t> q_off, q_idx, q_inv, kv_off, kv_idx, kv_inv, kv_slot_shard, vis;
+  std::vector<int32_t> kv_pos;  // position of every K/V row; empty = the row's own index
   std::vector<uint8_t> pair_class;
   std::vector<int4> qtiles[cascade::kNumTileSizes];
   void* dev_blob = nullptr;

@@ -1,5 +1,5 @@
 // Decode step with a token-sharded KV cache (Appendix F, "Caching"): one new query row per sequence against
-// every KV shard.  Each shard is an independent partial (Algorithm 3 with a single query row) and the K/V rows
+// every KV shard.  Each shard is an independent partial (the Attention-Pass algorithm with a single query row) and the K/V rows
 // of the cache are read exactly once, so the kernel must be bound by HBM reads of gathered 256-byte rows.
 //
 // One CTA = (KV shard, KV head, sequence); each of its 4 warps walks blocks of 16 gathered keys.  The G query

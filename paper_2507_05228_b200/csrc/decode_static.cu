@@ -71,6 +71,10 @@ extern "C" cascade_status_t cascade_attn_decode_static(const cascade_plan_t* pla
     set_error("cascade_attn_decode_static: bad batch or head counts");
     return CASCADE_ERR_INVALID_ARG;
   }
+  if (!(scale > 0.f) || scale > 3.0e38f) {
+    set_error("cascade_attn_decode_static: scale must be positive and finite");
+    return CASCADE_ERR_INVALID_ARG;
+  }
   const int G = n_kv_heads > 0 && n_heads % n_kv_heads == 0 ? n_heads / n_kv_heads : 0;
   if (plan->dev.n_q != 1 || !(G == 1 || G == 2 || G == 4 || G == 8)) {
     set_error("cascade_attn_decode_static: needs a plan with n_q == 1 and n_heads / n_kv_heads in {1,2,4,8} "

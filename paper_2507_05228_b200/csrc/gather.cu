@@ -1,15 +1,29 @@
 // Shard gather of the key/value rows (the paper's stage-A hand-over: every AttnNode receives k^{T_k}, v^{T_k}, the
-// rows of its KV shard in ascending token order, Algorithm 1 / Appendix D): copies K and V from token order into
+// rows of its KV shard in ascending token order, the Single Layer Forward Pass algorithm / Appendix D): copies K and V from token order into
 // shard-major order [batch][kv_head][slot][head_dim], slot = position in the plan's KV_IDX list.  After this pass
 // the visible prefix of a shard is a contiguous run of rows, which the attention kernel fetches with large TMA tile
 // loads; an index-mapped gather straight into shared memory could not feed the tensor cores (one 512-byte request
 // per ~36 cycles per SM with TMA row gathers, less with cp.async).  Bandwidth-bound: every K/V byte is read once
 // and written once, 16 bytes per thread.
+// Positions of a shard's list that no query row of the plan sees (keys later than the last query position: the unwritten
+// tail of a preallocated cache) are written as zeros instead of copied.  The attention kernel loads whole 16-key
+// chunks and multiplies the rows past a prefix by zero weights, so what it loads there must be finite, whatever the
+// caller's tensors hold at those positions.
 #include "cascade_internal.cuh"
 
 namespace cascade {
 
 constexpr int kGatherRowsPerCta = 64;
+
+// True if position `slot` of the shard-major order lies inside the longest visible prefix of its shard, i.e. the
+// prefix seen by the query row with the largest position (the last token of the query block).
+__device__ __forceinline__ bool slot_is_visible(const PlanDev& pl, int map, int slot) {
+  const int P = pl.n_kv_shards;
+  const int kk = __ldg(pl.kv_slot_shard + (size_t)map * pl.n_kv + slot);
+  const int last_slot = __ldg(pl.q_inv + (size_t)map * pl.n_q + pl.n_q - 1);
+  const int longest = __ldg(pl.vis + ((size_t)map * pl.n_q + last_slot) * P + kk);
+  return slot - __ldg(pl.kv_off + (size_t)map * (P + 1) + kk) < longest;
+}
 
 __global__ void __launch_bounds__(256) gather_kv_kernel(AttnParams p, __nv_bfloat16* k_out, __nv_bfloat16* v_out) {
   constexpr int D = 128;
@@ -29,7 +43,8 @@ __global__ void __launch_bounds__(256) gather_kv_kernel(AttnParams p, __nv_bfloa
 #pragma unroll
   for (int i = 0; i < kGatherRowsPerCta / 16; ++i) {
     const int slot = slot0 + 16 * i + r0;
-    if (slot < pl.n_kv) {
+    kr[i] = vr[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (slot < pl.n_kv && slot_is_visible(pl, map, slot)) {
       const int64_t tok = __ldg(kv_idx + slot);
       kr[i] = __ldcs(reinterpret_cast<const uint4*>(kb + tok * p.ks.token + chunk * 8));
       vr[i] = __ldcs(reinterpret_cast<const uint4*>(vb + tok * p.vs.token + chunk * 8));
@@ -60,7 +75,7 @@ __device__ __forceinline__ void rotate8(uint4& lo, uint4& hi, const float2* __re
   }
 }
 
-// The same gather with the rotary step of the pre-pass (Algorithm 2: k <- rotary_pos_emb(k, p^{R_i})) applied to the
+// The same gather with the rotary step of the pre-pass (the Pre-Pass algorithm: k <- rotary_pos_emb(k, p^{R_i})) applied to the
 // key rows on the way: a key row is turned by the angles of its own token index, so the rotation needs nothing but
 // the row and its row of the positional table.  A thread holds both halves of 8 rotation pairs (columns 8c.. and
 // 64 + 8c..), 8 threads per row; V rows are copied as they are.
@@ -82,7 +97,9 @@ __global__ void __launch_bounds__(256) gather_kv_rope_kernel(AttnParams p, __nv_
 #pragma unroll
   for (int i = 0; i < kPasses; ++i) {
     const int slot = slot0 + 32 * i + r0;
-    if (slot < pl.n_kv) {
+    klo[i] = khi[i] = vlo[i] = vhi[i] = make_uint4(0u, 0u, 0u, 0u);
+    tok[i] = -1;
+    if (slot < pl.n_kv && slot_is_visible(pl, map, slot)) {
       tok[i] = __ldg(kv_idx + slot);
       const __nv_bfloat16* kr = kb + (int64_t)tok[i] * p.ks.token + chunk * 8;
       const __nv_bfloat16* vr = vb + (int64_t)tok[i] * p.vs.token + chunk * 8;
@@ -96,7 +113,7 @@ __global__ void __launch_bounds__(256) gather_kv_rope_kernel(AttnParams p, __nv_
   for (int i = 0; i < kPasses; ++i) {
     const int slot = slot0 + 32 * i + r0;
     if (slot < pl.n_kv) {
-      rotate8(klo[i], khi[i], p.rope + (int64_t)tok[i] * (D / 2) + chunk * 8);
+      if (tok[i] >= 0) rotate8(klo[i], khi[i], p.rope + (int64_t)tok[i] * (D / 2) + chunk * 8);
       __nv_bfloat16* ko = k_out + (out_base + slot) * D + chunk * 8;
       __nv_bfloat16* vo = v_out + (out_base + slot) * D + chunk * 8;
       *reinterpret_cast<uint4*>(ko) = klo[i];
@@ -120,7 +137,7 @@ cudaError_t launch_gather_kv(const AttnParams& p, void* k_out, void* v_out, cuda
   return cudaGetLastError();
 }
 
-// Positional table p of the rotary embedding (Section 4: p is set up before inference; Algorithm 2 takes its rows
+// Positional table p of the rotary embedding (Section 5.1: p is set up before inference; the Pre-Pass algorithm takes its rows
 // p^{R_i}): table[t * d/2 + i] = (cos, sin)(t * base^(-2 i / d)), angles formed and evaluated in fp64, stored as fp32.
 __global__ void __launch_bounds__(256) rope_table_kernel(int32_t n_positions, int32_t half, double base,
                                                          float2* __restrict__ table) {

@@ -1,4 +1,4 @@
-// Post-pass combine (Algorithm 4 lines 1-8): a log-sum-exp weighted average of the per-shard partials.
+// Post-pass combine (the Post-Pass algorithm): a log-sum-exp weighted average of the per-shard partials.
 // Bandwidth-bound: every partial is read exactly once with 16-byte loads; one thread owns 16 bytes of one
 // (row, head) output vector and loops over the parts with several loads in flight.
 #include "cascade_internal.cuh"
@@ -74,7 +74,7 @@ __global__ void __launch_bounds__(256, 8) merge_kernel(MergeParams p) {
   const float* lp = p.l_part + (int64_t)b * P * part_stride + rh;
   const T* up = static_cast<const T*>(p.o_part) + ((int64_t)b * P * part_stride + rh) * D + sub * V;
 
-  // line 3: n = max over parts of m
+  // n = max over parts of m
   float n = -INFINITY;
   for (int k = sub; k < P; k += TPR) n = fmaxf(n, __ldg(mp + (int64_t)k * part_stride));
 #pragma unroll
@@ -85,7 +85,7 @@ __global__ void __launch_bounds__(256, 8) merge_kernel(MergeParams p) {
   for (int i = 0; i < V; ++i) acc[i] = 0.f;
   float w = 0.f;
   for (int base = 0; base < P; base += TPR) {
-    // lines 5-6: weight exp(m_k - n) * l_k of part base + sub (an empty part has l = 0)
+    // weight exp(m_k - n) * l_k of part base + sub (an empty part has l = 0)
     float wt = 0.f;
     if (base + sub < P) {
       const float mk = __ldg(mp + (int64_t)(base + sub) * part_stride);
@@ -110,7 +110,7 @@ __global__ void __launch_bounds__(256, 8) merge_kernel(MergeParams p) {
 #pragma unroll
   for (int off = TPR / 2; off > 0; off >>= 1) w += __shfl_xor_sync(0xffffffffu, w, off);
   if (!active) return;
-  const float inv = w > 0.f ? 1.f / w : 0.f;  // line 8
+  const float inv = w > 0.f ? 1.f / w : 0.f;  // the final division by w
 #pragma unroll
   for (int i = 0; i < V; ++i) acc[i] *= inv;
   const int out_row = p.row_scatter ? __ldg(p.row_scatter + (int64_t)b * p.row_scatter_batch_stride + r) : r;

@@ -141,9 +141,11 @@ def config(name: str, **overrides) -> Workload:
     return make_workload(name, **kw)
 
 
-def sample_rows(w: Workload, per_shard: int, seed: int = 1234) -> np.ndarray:
+def sample_rows(w: Workload, per_shard: int, seed: int = 1234, tile_edges: bool = False) -> np.ndarray:
     """A seeded sample of query rows (token ids), stratified over query shards: the first and last token of
-    every shard plus ``per_shard`` random members, ascending and unique."""
+    every shard plus ``per_shard`` random members, ascending and unique.  With ``tile_edges`` also the members at
+    the positions of a shard's list where kernels change tile or sub-tile: 31, 32, 63, 64, 127 and the first of
+    every group of 128."""
     rng = np.random.Generator(np.random.PCG64(seed))
     picked = []
     for j in range(w.n_q_shards):
@@ -151,5 +153,8 @@ def sample_rows(w: Workload, per_shard: int, seed: int = 1234) -> np.ndarray:
         if members.size == 0:
             continue
         picked += [members[0], members[-1]]
+        if tile_edges:
+            slots = [s for s in (31, 32, 63, 64, 127) if s < members.size] + list(range(0, members.size, 128))
+            picked += list(members[slots])
         picked += list(rng.choice(members, size=min(per_shard, members.size), replace=False))
     return np.unique(np.asarray(picked, dtype=np.int32))

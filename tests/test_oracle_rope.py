@@ -1,4 +1,4 @@
-"""Pins for the rotary step of the oracle (Algorithm 2, last two steps), against what the mathematics fixes:
+"""Pins for the rotary step of the oracle (the rotary steps of the Pre-Pass algorithm), against what the mathematics fixes:
 textbook values, the rotation group law, the relative-position property and an independent complex-number route."""
 import numpy as np
 
@@ -92,7 +92,7 @@ def test_rounding_to_bf16_straight_from_fp64():
 
 
 def test_rotation_commutes_with_sharding():
-    # rows rotated shard by shard with p^{R_i} equal the rows of the whole sequence rotated with p (Algorithm 2
+    # rows rotated shard by shard with p^{R_i} equal the rows of the whole sequence rotated with p (the Pre-Pass algorithm
     # takes the positions of the node's own index set), and sharded attention on them equals unsharded attention
     B, n, H, Hkv, d, base = 1, 24, 2, 1, 8, 10000.0
     rng = np.random.default_rng(6)

@@ -33,7 +33,9 @@ def test_c3_batched_reduced_and_outliers(gu):
 
 
 def test_c3_batched_full_size_sampled(gu):
-    gu.sampled_parity(wl.config("c3_batched"), per_shard=1)
+    """Full size, in the launch configuration the benchmark times; at least 1024 query rows (every batch entry, all
+    heads) go through the oracle."""
+    gu.sampled_parity(wl.config("c3_batched"), per_shard=56, min_rows=1024)
 
 
 def test_c4_long_reduced(gu):
@@ -41,7 +43,15 @@ def test_c4_long_reduced(gu):
 
 
 def test_c4_long_full_size_sampled(gu):
-    gu.sampled_parity(wl.config("c4_long_70b"), per_shard=1)
+    gu.sampled_parity(wl.config("c4_long_70b"), per_shard=19, min_rows=1024)
+
+
+def test_all_rows_in_the_grid_order_of_large_problems(gu):
+    """More CTAs than eight per SM switch the tensor-core kernel to its other block-index decoding (head group
+    slowest); every row of such a launch goes through the oracle."""
+    w = wl.config("c2_prefill_8b", B=3, n_q=4096, n_kv=4096)
+    assert (4096 // 64) * (w.H // 4) * w.B > 8 * 148
+    gu.full_parity(w)
 
 
 def test_c5_decode_full(gu):
@@ -118,7 +128,7 @@ def test_per_sequence_maps_and_strided_inputs(gu):
     o_m, _ = cb.cascade_merge(o_part, m_part, l_part, plan.dev_ptr("q_idx"), row_scatter_batch_stride=n)
     o_f, lse_f = cb.cascade_attn_sharded(plan, qv, kv, vv, w.scale)
     o_ref, lse_ref = oracle.attention_unsharded(w.q, w.k, w.v, w.scale)
-    gu.check_output(o_m, None, o_ref, lse_ref, w.tol, "per-sequence maps merge")
+    gu.check_output(o_m, None, o_ref, lse_ref, w.tol, "per-sequence maps merge", stored_partials=True)
     gu.check_output(o_f, lse_f, o_ref, lse_ref, w.tol, "per-sequence maps fused")
     for b in range(B):
         op = oracle.shard_plan(maps[b], maps[b], 4, 4)
@@ -258,3 +268,46 @@ def test_decode_loop_over_a_preallocated_cache_with_plan_advance(gu):
     assert plan.device_status() == 0 and plan2.device_status() == 0
     plan.destroy()
     plan2.destroy()
+
+
+@pytest.mark.parametrize("dtype,d,n_q", [("bf16", 128, 64), ("bf16", 128, 1), ("f32", 64, 48)])
+def test_unwritten_cache_tail_may_hold_nan(gu, dtype, d, n_q):
+    """A preallocated cache whose rows beyond the last query position were never written (NaN bit patterns here) must not
+    leak into the result on any route: tensor cores (whole 32-key chunks are loaded, rows past a prefix get weight 0,
+    and 0 x NaN would poison the output), decode and the ALU kernel."""
+    from paper_2507_05228_b200 import binding as cb
+    cap, B, H, Hkv, P = 512, 2, 8, 2, 4
+    w = wl.make_workload("nan_tail", B, n_q, cap, H, Hkv, d, dtype, "round_robin", "block_rr", 2 if n_q > 1 else 1, P,
+                         seed=51, block=8, q_pos_offset=0)
+    q, k, v = gu.to_device(w)
+    plan = gu.make_plan(w)
+    for off in (0, 100, cap - n_q):
+        plan.advance(off)
+        last = off + n_q - 1
+        k_p, v_p = k.clone(), v.clone()
+        if last + 1 < cap:
+            k_p[:, last + 1:] = float("nan")
+            v_p[:, last + 1:] = float("nan")
+        o_ref, lse_ref = oracle.attention_unsharded(w.q, w.k, w.v, w.scale, causal=True, q_pos_offset=off)
+        o, lse = cb.cascade_attn_sharded(plan, q, k_p, v_p, w.scale)
+        gu.check_output(o, lse, o_ref, lse_ref, w.tol, f"fused, NaN tail after position {last}")
+        o_part, m_part, l_part = cb.cascade_attn_partials(plan, q, k_p, v_p, w.scale)
+        assert torch.isfinite(o_part.float()).all() and not torch.isnan(m_part).any() and torch.isfinite(l_part).all()
+        o_m, lse_m = cb.cascade_merge(o_part, m_part, l_part, plan.dev_ptr("q_idx"))
+        gu.check_output(o_m, lse_m, o_ref, lse_ref, w.tol, f"merge, NaN tail after position {last}",
+                        stored_partials=True)
+    assert plan.device_status() == 0
+    plan.destroy()
+
+
+def test_scale_must_be_positive_and_finite(gu):
+    from paper_2507_05228_b200 import binding as cb
+    w = wl.make_workload("scale", 1, 64, 64, 4, 2, 128, "bf16", "random", "random", 2, 2, seed=52)
+    q, k, v = gu.to_device(w)
+    plan = gu.make_plan(w)
+    for bad in (0.0, -0.5, float("inf"), float("nan")):
+        for call in (cb.cascade_attn_sharded, cb.cascade_attn_partials):
+            with pytest.raises(cb.CascadeError) as ei:
+                call(plan, q, k, v, bad)
+            assert ei.value.status == 1
+    plan.destroy()

@@ -118,3 +118,51 @@ def test_plan_advance_matches_a_plan_built_at_that_position(binding):
     plan.advance(40)
     assert np.array_equal(plan.get("vis"), before)
     plan.destroy()
+
+
+def test_resident_plans_are_the_columns_of_the_full_plan(binding):
+    """A party that keeps only the K/V rows of its own shards (every world-th shard): the plan over those rows, with
+    their original positions, must be the full plan restricted to those shards - lists re-indexed to the resident
+    rows, prefix lengths and pair classes copied.  Checked against the oracle's plan of the whole sequence, also
+    after moving the query block (cascade_plan_advance) and for a bidirectional mask."""
+    from paper_2507_05228_b200 import exchange as ex
+    rng = np.random.Generator(np.random.PCG64(77))
+    for trial in range(24):
+        n_q, n_kv = int(rng.integers(1, 200)), int(rng.integers(8, 260))
+        J, P = int(rng.integers(1, 6)), int(rng.integers(2, 9))
+        world = int(rng.integers(1, P + 1))
+        q_of = rng.integers(0, J, n_q).astype(np.int32)
+        kv_of = rng.integers(0, P, n_kv).astype(np.int32)
+        causal = bool(trial % 5)
+        off = int(rng.integers(-3, n_kv))
+        ref = oracle.shard_plan(q_of, kv_of, J, P, q_pos_offset=off, causal=causal)
+        for rank in range(world):
+            tokens, local_of, n_local = ex.resident_kv(kv_of, P, rank, world)
+            mine = ex.owned_shards(P, rank, world)
+            assert n_local == mine.size
+            if tokens.size == 0:
+                continue  # a plan needs at least one K/V row
+            plan = binding.cascade_shard_plan_resident(q_of, local_of, tokens, J, n_local, q_pos_offset=off,
+                                                       causal=causal, host_only=True)
+            assert np.array_equal(plan.get("q_idx")[0], ref.q_idx) and np.array_equal(plan.get("q_off")[0], ref.q_off)
+            assert np.array_equal(plan.get("vis")[0], ref.vis[:, mine])
+            assert np.array_equal(plan.get("pair_class")[0], ref.pair_class[:, mine])
+            # the lists hold resident-row indices; through `tokens` they are the full plan's lists of those shards
+            kv_off, kv_idx = plan.get("kv_off")[0], plan.get("kv_idx")[0]
+            for i, k in enumerate(mine):
+                assert np.array_equal(tokens[kv_idx[kv_off[i]:kv_off[i + 1]]], ref.kv_idx[ref.kv_off[k]:ref.kv_off[k + 1]])
+            new_off = off + 7
+            plan.advance(new_off)
+            ref2 = oracle.shard_plan(q_of, kv_of, J, P, q_pos_offset=new_off, causal=causal)
+            assert np.array_equal(plan.get("vis")[0], ref2.vis[:, mine])
+            assert np.array_equal(plan.get("pair_class")[0], ref2.pair_class[:, mine])
+            plan.destroy()
+
+
+def test_resident_plan_rejects_unordered_positions(binding):
+    q_of = np.zeros(4, np.int32)
+    kv_of = np.zeros(3, np.int32)
+    for bad in ([0, 2, 2], [3, 1, 5], [-1, 0, 1]):
+        with pytest.raises(binding.CascadeError) as ei:
+            binding.cascade_shard_plan_resident(q_of, kv_of, np.array(bad, np.int32), 1, 1, host_only=True)
+        assert ei.value.status == 2

@@ -1,4 +1,4 @@
-"""GPU parity of the fused rotary step (Algorithm 2's last two steps inside the staging of Q and K rows) against the
+"""GPU parity of the fused rotary step (the rotary steps of the Pre-Pass algorithm inside the staging of Q and K rows) against the
 fp64 oracle: the positional table, the rotated key rows left in the workspace, and the attention output.
 
 Tolerances: the table is fp32 of an fp64 evaluation (|err| <= 2^-24 + angle error); rotated key rows are computed in

@@ -37,6 +37,41 @@ def test_decode_static_matches_workspace_path_on_two_calls_in_a_row():
         plan.destroy()
 
 
+def test_decode_static_allocates_no_device_memory():
+    """After a first call (which loads the module and looks the scratch array up), a raw C-ABI call with outputs the
+    caller already owns leaves the device's free memory and torch's allocator exactly where they were."""
+    import gpu_util as gu
+    from paper_2507_05228_b200 import binding as cb
+
+    L = cb.lib()
+    S = cb._strides
+    w = wl.make_workload("static_mem", 4, 1, 1024, 16, 4, 128, "bf16", "round_robin", "random", 1, 8, seed=44)
+    q, k, v = gu.to_device(w)
+    plan = gu.make_plan(w)
+    o = torch.empty_like(q)
+    lse = torch.empty((w.B, 1, w.H), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def call():
+        rc = L.cascade_attn_decode_static(plan.handle, w.B, w.H, w.Hkv, w.scale, q.data_ptr(), S(q), k.data_ptr(), S(k),
+                                          v.data_ptr(), S(v), o.data_ptr(), S(o), lse.data_ptr(), stream)
+        assert rc == 0, L.cascade_last_error()
+
+    call()  # warm-up: module load, address look-up
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0, (free0, free1)
+    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+    o_ref, lse_ref = oracle.attention_unsharded(w.q, w.k, w.v, w.scale, q_pos_offset=w.q_pos_offset)
+    gu.check_output(o, lse, o_ref, lse_ref, w.tol, "static scratch, raw call")
+    plan.destroy()
+
+
 def test_decode_static_rejects_oversized_and_unsupported_problems():
     import gpu_util as gu
     from paper_2507_05228_b200 import binding as cb
