@@ -378,7 +378,52 @@ cascade_status_t cascade_attn_decode_static(const cascade_plan_t* plan, int32_t 
                                             cascade_strides_t v_strides, void* o_out, cascade_strides_t o_strides,
                                             float* lse_out, void* stream);
 
-enum { CASCADE_CALL_PARTIALS = 0, CASCADE_CALL_SHARDED = 1, CASCADE_CALL_SHARDED_HOST = 2 };
+/*
+ * cascade_rope_apply -- the rotary steps of the Pre-Pass algorithm (q <- rotary_pos_emb(q, p^{R_i}), the same for k) as
+ * a pass of its own, for rows that no fused call covers (fp32, head_dim 64, rows rotated once and then cached):
+ *   y[b][r][h][i]       = x[..][i] cos - x[..][i + d/2] sin
+ *   y[b][r][h][i + d/2] = x[..][i + d/2] cos + x[..][i] sin,      (cos, sin) = table[first_position + r][i]
+ * in fp32, rounded once to `dtype`.  Row r of every sequence sits at position first_position + r.
+ *   x, y         DEVICE [batch][n_rows][n_heads][head_dim] with strides (y may be x: in place); head_dim 64 or 128
+ *   rope_table   DEVICE table of cascade_rope_table for this head_dim; n_positions its row count
+ * Errors: INVALID_ARG (null, misaligned, positions outside the table), UNSUPPORTED (dtype, head_dim), CUDA.
+ */
+cascade_status_t cascade_rope_apply(cascade_dtype_t dtype, int32_t batch, int32_t n_rows, int32_t n_heads,
+                                    int32_t head_dim, const void* x, cascade_strides_t x_strides,
+                                    int32_t first_position, const float* rope_table, int32_t n_positions, void* y,
+                                    cascade_strides_t y_strides, void* stream);
+
+/*
+ * cascade_decode_step_rope -- one generated token against a token-sharded KV cache ("Caching" in the appendix on cost
+ * optimizations), with the tail of the Pre-Pass algorithm folded in: given the new token's UNROTATED q, k, v rows
+ *   1. moves the plan's query block to `position` (cascade_plan_advance: the mask admits cache rows <= position),
+ *   2. rotates the k row by the table row of `position` and writes it, and the v row as it is, at row `position` of the
+ *      caches -- the node that holds the token's KV shard appends it; rows already cached are not touched again,
+ *   3. rotates the q row and runs the decode route of cascade_attn_sharded on the caches (one partial per KV shard,
+ *      then the post-pass combine).
+ *   plan            built by cascade_shard_plan over the cache CAPACITY with n_q = 1 (see cascade_plan_advance)
+ *   q_new           DEVICE bf16 [batch][1][n_heads][128];  k_new, v_new  DEVICE bf16 [batch][1][n_kv_heads][128]
+ *   k_cache, v_cache  DEVICE bf16 [batch][capacity][n_kv_heads][128] with strides; row `position` is WRITTEN
+ *   rope_table      DEVICE table of cascade_rope_table for head_dim 128 with more than `position` rows
+ *   o_out, lse_out  as cascade_attn_sharded (one row per sequence)
+ *   workspace       cascade_workspace_bytes(CASCADE_CALL_DECODE_STEP_ROPE) bytes
+ * bf16, head_dim 128, n_heads / n_kv_heads in {1, 2, 4, 8}.  Errors as cascade_attn_sharded and cascade_plan_advance.
+ */
+cascade_status_t cascade_decode_step_rope(cascade_plan_t* plan, int32_t batch, int32_t n_heads, int32_t n_kv_heads,
+                                          float scale, const void* q_new, cascade_strides_t q_strides,
+                                          const void* k_new, cascade_strides_t k_new_strides, const void* v_new,
+                                          cascade_strides_t v_new_strides, void* k_cache,
+                                          cascade_strides_t k_cache_strides, void* v_cache,
+                                          cascade_strides_t v_cache_strides, int32_t position, const float* rope_table,
+                                          int32_t n_positions, void* o_out, cascade_strides_t o_strides, float* lse_out,
+                                          void* workspace, size_t workspace_bytes, void* stream);
+
+enum {
+  CASCADE_CALL_PARTIALS = 0,
+  CASCADE_CALL_SHARDED = 1,
+  CASCADE_CALL_SHARDED_HOST = 2,
+  CASCADE_CALL_DECODE_STEP_ROPE = 3
+};
 
 /* Scratch bytes the given call needs for this plan and shape (0 if none).  The workspace must be
  * 256-byte aligned. */

@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libcascade_b200.so")
 
 F32, BF16 = 0, 1
 CALL_PARTIALS, CALL_SHARDED = 0, 1
+CALL_DECODE_STEP_ROPE = 3
 PLAN_FIELDS = {"q_off": 0, "q_idx": 1, "q_inv": 2, "kv_off": 3, "kv_idx": 4, "kv_inv": 5, "vis": 6,
                "pair_class": 7}
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_MAP", 3: "UNSUPPORTED", 4: "WORKSPACE", 5: "ALLOC", 6: "CUDA",
@@ -31,7 +32,7 @@ EXPORTS = [
     "cascade_kernel_timing_begin", "cascade_kernel_timing_end", "cascade_rope_table", "cascade_attn_sharded_rope",
     "cascade_cdelta_shard_map", "cascade_msplit_shard_map", "cascade_index_set_gaps", "cascade_kl_gaps",
     "cascade_attn_sharded_host", "cascade_plan_advance", "cascade_shard_plan_resident",
-    "cascade_shard_plan_resident_host",
+    "cascade_shard_plan_resident_host", "cascade_rope_apply", "cascade_decode_step_rope",
 ]
 
 
@@ -65,6 +66,9 @@ def lib() -> ctypes.CDLL:
         L.cascade_shard_plan_host.argtypes = [i32, i32, i32, vp, vp, i32, i32, i32, i32, ctypes.POINTER(vp)]
         L.cascade_shard_plan_resident.argtypes = [i32, i32, i32, vp, vp, vp, i32, i32, i32, i32, vp, ctypes.POINTER(vp)]
         L.cascade_shard_plan_resident_host.argtypes = [i32, i32, i32, vp, vp, vp, i32, i32, i32, i32, ctypes.POINTER(vp)]
+        L.cascade_rope_apply.argtypes = [i32, i32, i32, i32, i32, vp, Strides, i32, vp, i32, vp, Strides, vp]
+        L.cascade_decode_step_rope.argtypes = [vp, i32, i32, i32, f32, vp, Strides, vp, Strides, vp, Strides, vp, Strides,
+                                               vp, Strides, i32, vp, i32, vp, Strides, vp, vp, ctypes.c_size_t, vp]
         L.cascade_plan_destroy.argtypes = [vp]
         L.cascade_plan_get.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(i64)]
         L.cascade_plan_dense_mask.argtypes = [vp, i32, i32, i32, vp, i64]
@@ -342,6 +346,35 @@ def cascade_attn_sharded_rope(plan: Plan, q: torch.Tensor, k: torch.Tensor, v: t
 
 
 CALL_SHARDED_HOST = 2
+
+
+def cascade_rope_apply(x: torch.Tensor, first_position: int, rope_table: torch.Tensor, out=None) -> torch.Tensor:
+    """The rotary steps of the pre-pass on x [B, n_rows, heads, d] (row r at position first_position + r); out may be x."""
+    B, n_rows, H, d = x.shape
+    y = out if out is not None else torch.empty_like(x)
+    _check(lib().cascade_rope_apply(_dtype_code(x), B, n_rows, H, d, x.data_ptr(), _strides(x), int(first_position),
+                                    rope_table.data_ptr(), rope_table.shape[0], y.data_ptr(), _strides(y), _stream()))
+    return y
+
+
+def cascade_decode_step_rope(plan: Plan, q_new: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
+                             k_cache: torch.Tensor, v_cache: torch.Tensor, position: int, scale: float,
+                             rope_table: torch.Tensor, out=None, want_lse: bool = True, workspace=None):
+    """One decode step over a token-sharded cache: advances the plan to `position`, appends the new token's rotated k
+    row and its v row to the caches, rotates q and runs decode + merge.  Returns (o [B, 1, H, 128], lse or None)."""
+    B, _, H, d = q_new.shape
+    Hkv = k_new.shape[2]
+    o = out if out is not None else torch.empty_like(q_new)
+    lse = torch.empty((B, 1, H), dtype=torch.float32, device=q_new.device) if want_lse else None
+    nbytes = cascade_workspace_bytes(plan, CALL_DECODE_STEP_ROPE, BF16, B, H, Hkv, d)
+    ws, ws_ptr, ws_bytes = _ws(nbytes, q_new.device, workspace)
+    _check(lib().cascade_decode_step_rope(plan.handle, B, H, Hkv, scale, q_new.data_ptr(), _strides(q_new),
+                                          k_new.data_ptr(), _strides(k_new), v_new.data_ptr(), _strides(v_new),
+                                          k_cache.data_ptr(), _strides(k_cache), v_cache.data_ptr(), _strides(v_cache),
+                                          int(position), rope_table.data_ptr(), rope_table.shape[0], o.data_ptr(),
+                                          _strides(o), lse.data_ptr() if lse is not None else None, ws_ptr, ws_bytes,
+                                          _stream()))
+    return o, lse
 
 
 def cascade_attn_sharded_host(plan: Plan, q_host: torch.Tensor, k_host: torch.Tensor, v_host: torch.Tensor,

@@ -42,6 +42,10 @@
 
 #include "cascade_internal.cuh"
 
+#ifndef CASCADE_PARTIALS_WALK
+#define CASCADE_PARTIALS_WALK 1
+#endif
+
 namespace cascade {
 namespace tc {
 
@@ -82,9 +86,10 @@ enum Bar {
   V_EMPTY = V_FULL + kVStages,    // [kVStages]
   S_FULL = V_EMPTY + kVStages,    // [2]
   P_FULL = S_FULL + 2,            // [2]
-  O_FULL = P_FULL + 2             // [1]
+  O_FULL = P_FULL + 2,            // [1]
+  O_RDY = O_FULL + 1              // [2]  kWalk: the accumulator of a sub-tile holds a finished shard
 };
-static_assert(O_FULL + 1 <= kNumBars, "barrier table too small");
+static_assert(O_RDY + 2 <= kNumBars, "barrier table too small");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -306,13 +311,47 @@ struct ChunkCursor {
   }
 };
 
+// Chunk count and shard-start flag of consecutive tiles, for the roles that do not walk the chunks themselves.
+template <bool kWalk>
+struct TileSeq {
+  const ShardTab* t;
+  int n_act, n_chunks, i, j, c, nc;
+  __device__ __forceinline__ TileSeq(const ShardTab* tab, int n_active, int chunks)
+      : t(tab), n_act(n_active), n_chunks(chunks), i(0), j(0), c(0) {
+    nc = (kWalk && n_act > 0) ? (t->need[0] + kChunk - 1) / kChunk : 0;
+  }
+  // the next tile: its chunks; first = it opens a shard (kWalk) or the whole stream
+  __device__ __forceinline__ int next(bool& first) {
+    if constexpr (!kWalk) {
+      first = i == 0;
+      const int n = min(4, n_chunks - 4 * i);
+      ++i;
+      return n;
+    } else {
+      first = c == 0;
+      const int n = min(4, nc - c);
+      c += n;
+      if (c >= nc) {
+        ++j;
+        c = 0;
+        nc = j < n_act ? (t->need[j] + kChunk - 1) / kChunk : 0;
+      }
+      return n;
+    }
+  }
+};
+
 struct TmaArgs {
   CUtensorMap k, v;  // shard-major copies as [batch * kv_heads][n_kv][head_dim]
 };
 
 // kRope: the query rows are turned by the rotary embedding of their positions while they are staged (the key rows
 // were turned by the gather pass), the Pre-Pass algorithm.
-template <bool kRope>
+// kWalk: the partials of EVERY KV shard for one query tile in one CTA (the attention-pass of the nodes AttnNode_{j,1..beta}
+// one after another): the shards are walked as in the fused mode, but a tile never mixes two shards, and at a shard
+// boundary the softmax threads write that shard's (u, m, l) out and start over.  The query tile, the TMEM allocation,
+// the barriers and the K/V pipelines are set up once per query tile instead of once per (query tile, KV shard).
+template <bool kRope, bool kWalk>
 __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_constant__ AttnParams p, int lg,
                                                               int tile_major,
                                                               const __grid_constant__ TmaArgs tma) {
@@ -331,7 +370,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   const int Gp = 1 << lg, R = kM >> lg;
   const PlanDev& pl = p.plan;
   const int P = pl.n_kv_shards;
-  const int n_parts = p.fused ? 1 : P;
+  const int n_parts = (p.fused || kWalk) ? 1 : P;
   // CTA index -> (query tile, batch, part, head group).  The tile lists are sorted by decreasing work.  With few CTAs
   // per SM the query tile is the slowest index, so that the heaviest CTAs of all heads and sequences start first and
   // the light ones fill the tail.  For a large problem the head group is slowest instead: the CTAs running at any
@@ -368,7 +407,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   const int32_t* q_idx = pl.q_idx + (size_t)map * pl.n_q;
   const int32_t* kv_off = pl.kv_off + (size_t)map * (P + 1);
   const int32_t* vis = pl.vis + (size_t)map * pl.n_q * P;
-  const int k_begin = p.fused ? 0 : part, k_end = p.fused ? P : part + 1;
+  const int k_begin = (p.fused || kWalk) ? 0 : part, k_end = (p.fused || kWalk) ? P : part + 1;
   // Query sub-tiles (row r = slot r / Gp, head r % Gp): the 128 softmax threads of a sub-tile gather it from the
   // caller's tensor, 16 bytes per thread and row, half a warp per 256-byte row.  The loads are issued here, before the
   // set-up below, and land in shared memory (128-byte-swizzled [2][128][128 B] layout) after it.  Rows past the end
@@ -431,6 +470,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       }
       n_act += __popc(act);
       int ch = (nd + kChunk - 1) / kChunk;
+      if (kWalk) ch = (ch + 3) >> 2;  // tiles of this shard: a tile does not continue into the next shard
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) ch += __shfl_xor_sync(0xffffffffu, ch, off);
       n_chunks += ch;
@@ -461,6 +501,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
       mbar_init(bar(P_FULL + s), 128);
     }
     mbar_init(bar(O_FULL), 1);
+    mbar_init(bar(O_RDY), 1);
+    mbar_init(bar(O_RDY + 1), 1);
     *abort_flag = 0;
     for (int w = 0; w < kThreads / 32; ++w) progress[w] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -477,9 +519,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const int n_act = stream_info[0];                 // shards of which the CTA sees something
-  const int n_chunks = stream_info[1];              // chunks of the KV stream
-  const int n_tiles = (n_chunks + 3) >> 2;          // MMA tiles: four chunks each, the last one possibly fewer
-  auto tile_chunks = [&](int i) { return min(4, n_chunks - 4 * i); };
+  const int n_chunks = stream_info[1];              // chunks of the KV stream (kWalk: tiles, counted per shard)
+  // MMA tiles: four chunks each; only the last one is narrower, or with kWalk the last one of every shard
+  const int n_tiles = kWalk ? n_chunks : (n_chunks + 3) >> 2;
+  auto tile_chunks = [&](int i) { return min(4, n_chunks - 4 * i); };  // not with kWalk: see TileSeq
 
   if (warp < 8) {
     // ------------------------------------------------------------------ softmax + epilogue
@@ -549,8 +592,60 @@ if constexpr (kRope) {
       int vq0 = row_vis(0), vq1 = row_vis(1), vq2 = row_vis(2), vq3 = row_vis(3);
       ChunkCursor cur;
       cur.start(tab, n_act);
+      int kk_open = -1;  // kWalk: the shard whose partial is being accumulated
+      int n_flushed = 0;  // kWalk: partials written so far
+      const bool rows32 = (reinterpret_cast<uintptr_t>(p.o_part) & 31) == 0;  // partial rows are 256 bytes apart
+      // kWalk: writes the finished partial of shard kk (this thread's row of u, and m, l) straight from TMEM and the
+      // running statistics, then starts over.  The row goes out as sixteen 16-byte stores.
+      auto flush_shard = [&](int kk) {
+        float o_scale = 0.f, m_out = -INFINITY, l_out = 0.f;
+        if (l_run > 0.f) {
+          o_scale = 1.f / l_run;
+          l_out = l_run * ex2(m_run - m_true);
+          m_out = m_true * 0.6931471805599453f;
+        }
+        const int64_t stat = (((int64_t)b * P + kk) * pl.n_q + slot) * p.H + head;
+        if (row_ok) {
+          p.m_part[stat] = m_out;
+          p.l_part[stat] = l_out;
+        }
+        __nv_bfloat16* dst0 = static_cast<__nv_bfloat16*>(p.o_part) + stat * kD;
+        // 64 columns per round trip, then 32-byte stores: a row's 16-byte pieces would half-fill 32 sectors per store
+        // instruction
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+        uint32_t o[64];
+        CASCADE_TMEM_LD32(o_addr + (uint32_t)(half * 64), o, 0);
+        CASCADE_TMEM_LD32(o_addr + (uint32_t)(half * 64 + 32), o, 32);
+        tmem_wait_ld();
+        if (row_ok) {
+          __nv_bfloat16* dst = dst0 + half * 64;
+#pragma unroll
+          for (int j = 0; j < 64; j += 16) {
+            uint32_t w[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              w[e] = pack_bf16x2(__uint_as_float(o[j + 2 * e]) * o_scale, __uint_as_float(o[j + 2 * e + 1]) * o_scale);
+            if (rows32) {
+              asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + j), "r"(w[0]),
+                           "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                           : "memory");
+            } else {
+              *reinterpret_cast<uint4*>(dst + j) = make_uint4(w[0], w[1], w[2], w[3]);
+              *reinterpret_cast<uint4*>(dst + j + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+            }
+          }
+        }
+        }
+        m_run = -INFINITY;
+        m_true = -INFINITY;
+        l_run = 0.f;
+      };
       for (int i = 0; i < n_tiles; ++i) {
-        const int nch = tile_chunks(i);
+        // kWalk: a tile holds chunks of one shard only; the cursor stands at the tile's first chunk
+        const int nch = kWalk ? min(4, cur.nc - cur.c) : tile_chunks(i);
+        const bool opens = kWalk ? cur.c == 0 : i == 0;  // first tile of a shard (kWalk) or of the stream
+        const int kk_tile = kWalk ? tab->kk[cur.j] : 0;
         // Mask bookkeeping for the tile's four chunks, done before the wait so that it costs nothing: a chunk of shard
         // j starting at key t0 needs the mask only if it reaches past the shortest prefix of the sub-tile; this row
         // then sees its first lc = vis - t0 columns.  Chunks a narrow last tile does not have count as fully masked.
@@ -574,6 +669,20 @@ if constexpr (kRope) {
           }
         }
         note(8 * i + 1);
+        if constexpr (kWalk) {
+          // The issuing warp commits O_RDY right after the last product of a shard, before it issues the logits of
+          // this tile, so the previous shard's partial is written out while those logits are computed.  The first
+          // product of this shard (which overwrites the accumulator) waits for this thread's arrival on P_FULL(i).
+          if (opens) {
+            if (i > 0) {
+              wait_bar(wc, bar(O_RDY + s), (uint32_t)(n_flushed & 1), 2, i);
+              tc_fence_after();
+              flush_shard(kk_open);
+              ++n_flushed;
+            }
+            kk_open = kk_tile;
+          }
+        }
         wait_bar(wc, bar(S_FULL + s), (uint32_t)(i & 1), 1, i);
         tc_fence_after();
         uint32_t sr[128];
@@ -653,7 +762,7 @@ if constexpr (kRope) {
         l_run = l_run * alpha + ((psum0 + psum1) + (p_top_seen - p_top));
         // S_FULL(i) was committed after PV(i-1), so the output accumulator is quiescent until this thread's
         // arrival on P_FULL(i) below
-        if (i > 0 && __any_sync(0xffffffffu, changed)) {
+        if (!opens && __any_sync(0xffffffffu, changed)) {
           // rescale this warp's 32 rows of the output accumulator
           const float f = changed ? alpha : 1.f;
 #pragma unroll
@@ -683,7 +792,8 @@ if constexpr (kRope) {
           dst = static_cast<__nv_bfloat16*>(p.o_out) + (int64_t)b * p.os.batch + (int64_t)tok * p.os.token +
                 (int64_t)head * p.os.head;
         } else {
-          stat = (((int64_t)b * P + part) * pl.n_q + slot) * p.H + head;
+          // kWalk: the last shard the CTA saw anything of; its other shards were written on the way
+          stat = (((int64_t)b * P + (kWalk ? max(kk_open, 0) : part)) * pl.n_q + slot) * p.H + head;
           dst = static_cast<__nv_bfloat16*>(p.o_part) + stat * kD;
         }
       }
@@ -736,6 +846,25 @@ if constexpr (kRope) {
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // the row has left shared memory
       }
+      if constexpr (kWalk) {
+        // the shards of which no row of the CTA sees anything were never walked: their partials are empty
+        if (row_ok) {
+          int a = 0;
+          for (int k = 0; k < P; ++k) {
+            if (a < n_act && tab->kk[a] == k) {
+              ++a;
+              continue;
+            }
+            if (n_act == 0 && k == 0) continue;  // written by the epilogue above
+            const int64_t st2 = (((int64_t)b * P + k) * pl.n_q + slot) * p.H + head;
+            p.m_part[st2] = -INFINITY;
+            p.l_part[st2] = 0.f;
+            uint4* row = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.o_part) + st2 * kD);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) row[j] = make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+      }
       tc_fence_before();
     }
   } else {
@@ -766,7 +895,8 @@ if constexpr (kRope) {
             mma_commit(bar(S_FULL + s));
           }
         };
-        auto issue_pv = [&](int s, int i, int n) {  // O_s (+)= P_s V(i) over n keys
+        // O_s (+)= P_s V(i) over n keys; a tile that opens a shard (kWalk) or the stream starts the accumulator afresh
+        auto issue_pv = [&](int s, int i, int n, bool opens) {
           const uint32_t v_lo = v_lo0 + (uint32_t)((i % kVStages) * (kTileBytes >> 4));
           const int ksteps = n >> 4;
           if (leader) {
@@ -775,28 +905,35 @@ if constexpr (kRope) {
               // A = P from TMEM: 16 keys = 8 columns; B = V (MN-major): 16 keys = 16 rows of 128 bytes
               if (ks < ksteps)
                 mma_ts(tmem + 256u + (uint32_t)(s * 128), tmem + (uint32_t)(s * 128 + ks * 8),
-                       v_lo + (uint32_t)(ks * (2048 >> 4)), hi_v, idesc_pv, i > 0 || ks > 0);
+                       v_lo + (uint32_t)(ks * (2048 >> 4)), hi_v, idesc_pv, !opens || ks > 0);
             }
           }
         };
+        TileSeq<kWalk> seq(tab, n_act, n_chunks);
+        bool opens_cur = true, opens_next = false;
+        int n_cur = kChunk * seq.next(opens_cur), n_next = 0;
         wait_bar(wc, bar(K_FULL), 0u, 7);
         for (int s = 0; s < n_sub; ++s) {
           wait_bar(wc, bar(Q_FULL + s), 0u, 6);
           tc_fence_after();
-          issue_qk(s, 0, kChunk * tile_chunks(0));
+          issue_qk(s, 0, n_cur);
         }
         if (leader) mma_commit(bar(K_EMPTY));
         for (int i = 0; i < n_tiles; ++i) {
           const bool has_next = i + 1 < n_tiles;
-          const int n_cur = kChunk * tile_chunks(i);
-          const int n_next = has_next ? kChunk * tile_chunks(i + 1) : 0;
+          if (i > 0) {
+            n_cur = n_next;
+            opens_cur = opens_next;
+          }
+          n_next = has_next ? kChunk * seq.next(opens_next) : 0;
           note(8 * i + 1);
           wait_bar(wc, bar(V_FULL + i % kVStages), (uint32_t)((i / kVStages) & 1), 4, i);
           for (int s = 0; s < n_sub; ++s) {
             note(8 * i + 2 + s);
             wait_bar(wc, bar(P_FULL + s), (uint32_t)(i & 1), 5, i);
             tc_fence_after();
-            issue_pv(s, i, n_cur);
+            issue_pv(s, i, n_cur, opens_cur);
+            if (kWalk && has_next && opens_next && leader) mma_commit(bar(O_RDY + s));
             if (s == n_sub - 1 && leader) mma_commit(bar(V_EMPTY + i % kVStages));
             if (has_next) {
               if (s == 0) {
@@ -834,7 +971,7 @@ if constexpr (kRope) {
         // (a no-op otherwise).  Nothing else in this kernel reads what the gather grid writes.
         asm volatile("griddepcontrol.wait;" ::: "memory");
         for (int i = 0; i < n_tiles; ++i) {
-          const int nch = tile_chunks(i);
+          const int nch = kWalk ? min(4, cur.nc - cur.c) : tile_chunks(i);
           const int st = i % n_stages;
           note(8 * i + 1);
           wait_bar(wc, bar(empty0 + st), (uint32_t)(((i / n_stages) & 1) ^ 1), is_k ? 9 : 10, i);
@@ -913,7 +1050,10 @@ int sm_count() {
 }  // namespace
 
 cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void* v_sorted, cudaStream_t stream) {
-  auto kernel = p.rope ? tc::attn_tc_kernel<true> : tc::attn_tc_kernel<false>;
+  // the unfused route walks all KV shards of a query tile in one CTA (CASCADE_PARTIALS_WALK=0: a CTA per pair)
+  const bool walk = !p.fused && CASCADE_PARTIALS_WALK && p.plan.n_kv_shards > 1;
+  auto kernel = p.rope ? tc::attn_tc_kernel<true, false>
+                       : (walk ? tc::attn_tc_kernel<false, true> : tc::attn_tc_kernel<false, false>);
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes);
   if (e != cudaSuccess) return e;
   tc::TmaArgs tma;
@@ -925,7 +1065,7 @@ cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void
   // stack as many of the G heads of a KV head into one MMA tile as divide G (at most 8)
   int lg = 0;
   while (lg < 3 && p.G % (2 << lg) == 0) ++lg;
-  const int n_parts = p.fused ? 1 : p.plan.n_kv_shards;
+  const int n_parts = (p.fused || walk) ? 1 : p.plan.n_kv_shards;
   const int64_t n_ctas = (int64_t)p.plan.n_qtiles[3 - lg] * (p.H >> lg) * p.batch * n_parts;
   if (n_ctas >= (int64_t)1 << 31) return cudaErrorInvalidConfiguration;
   const int tile_major = n_ctas <= 8 * (int64_t)sm_count();  // few CTAs per SM: balance matters more than L2 locality

@@ -645,9 +645,9 @@ struct HostCallStreams {
   bool ready = false;
   cudaStream_t h2d = nullptr, d2h = nullptr;
   cudaEvent_t start = nullptr, done = nullptr;
-  cudaEvent_t uploaded[kMaxHostGroups], computed[kMaxHostGroups];
+  std::vector<cudaEvent_t> uploaded, computed;  // one pair per head group, created when a call first needs it
 };
-static HostCallStreams g_host_streams[16];
+static HostCallStreams g_host_streams[64];
 
 }  // namespace cascade
 
@@ -672,6 +672,14 @@ cascade_status_t cascade_workspace_bytes(const cascade_plan_t* plan, int32_t whi
     *out_bytes = decode ? decode_ws_bytes(plan, dtype, batch, n_heads, head_dim) : tc_bytes;
   } else if (which_call == CASCADE_CALL_SHARDED_HOST) {
     *out_bytes = host_call_layout(plan, dtype, batch, n_heads, n_kv_heads, head_dim).total;
+  } else if (which_call == CASCADE_CALL_DECODE_STEP_ROPE) {
+    if (!decode) {
+      set_error("cascade_workspace_bytes: the decode step needs a plan with one query row, bf16, head_dim 128");
+      return CASCADE_ERR_UNSUPPORTED;
+    }
+    // the partials of the decode kernel, then the rotated query rows
+    *out_bytes = align_up(decode_ws_bytes(plan, dtype, batch, n_heads, head_dim), 256) +
+                 align_up((size_t)batch * n_heads * head_dim * elt_size(dtype), 256);
   } else {
     set_error("cascade_workspace_bytes: unknown call %d", which_call);
     return CASCADE_ERR_INVALID_ARG;
@@ -901,6 +909,100 @@ cascade_status_t cascade_rope_table(int32_t n_positions, int32_t head_dim, doubl
   return CASCADE_OK;
 }
 
+cascade_status_t cascade_rope_apply(cascade_dtype_t dtype, int32_t batch, int32_t n_rows, int32_t n_heads,
+                                    int32_t head_dim, const void* x, cascade_strides_t x_strides,
+                                    int32_t first_position, const float* rope_table, int32_t n_positions, void* y,
+                                    cascade_strides_t y_strides, void* stream) {
+  const char* fn = "cascade_rope_apply";
+  if (!x || !y || !rope_table) {
+    set_error("%s: null pointer", fn);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (dtype != CASCADE_F32 && dtype != CASCADE_BF16) {
+    set_error("%s: unknown dtype %d", fn, (int)dtype);
+    return CASCADE_ERR_UNSUPPORTED;
+  }
+  if (head_dim != 64 && head_dim != 128) {
+    set_error("%s: head_dim %d unsupported (64 or 128)", fn, head_dim);
+    return CASCADE_ERR_UNSUPPORTED;
+  }
+  if (batch < 1 || n_rows < 1 || n_heads < 1 || first_position < 0 ||
+      (int64_t)first_position + n_rows > (int64_t)n_positions) {
+    set_error("%s: sizes must be positive and positions %d .. %lld must lie inside the table of %d rows", fn,
+              first_position, (long long)first_position + n_rows - 1, n_positions);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  const size_t es = elt_size(dtype);
+  if (!aligned16(x) || !aligned16(y) || !aligned16(rope_table) || !strides_ok(x_strides, es) ||
+      !strides_ok(y_strides, es)) {
+    set_error("%s: pointers and row strides must be 16-byte aligned", fn);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  cudaError_t e = launch_rope_apply(dtype, batch, n_rows, n_heads, head_dim, x,
+                                    {x_strides.batch, x_strides.token, x_strides.head}, first_position,
+                                    reinterpret_cast<const float2*>(rope_table), y,
+                                    {y_strides.batch, y_strides.token, y_strides.head}, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e, "cascade_rope_apply: launch");
+  return CASCADE_OK;
+}
+
+cascade_status_t cascade_decode_step_rope(cascade_plan_t* plan, int32_t batch, int32_t n_heads, int32_t n_kv_heads,
+                                          float scale, const void* q_new, cascade_strides_t q_strides,
+                                          const void* k_new, cascade_strides_t k_new_strides, const void* v_new,
+                                          cascade_strides_t v_new_strides, void* k_cache,
+                                          cascade_strides_t k_cache_strides, void* v_cache,
+                                          cascade_strides_t v_cache_strides, int32_t position, const float* rope_table,
+                                          int32_t n_positions, void* o_out, cascade_strides_t o_strides, float* lse_out,
+                                          void* workspace, size_t workspace_bytes, void* stream) {
+  const char* fn = "cascade_decode_step_rope";
+  constexpr int kHeadDim = 128;
+  if (!plan || !q_new || !k_new || !v_new || !k_cache || !v_cache || !rope_table || !o_out) {
+    set_error("%s: null pointer", fn);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  cascade_status_t s = check_attn_args(fn, plan, CASCADE_BF16, batch, n_heads, n_kv_heads, kHeadDim, scale, q_new,
+                                       q_strides, k_cache, k_cache_strides, v_cache, v_cache_strides);
+  if (s != CASCADE_OK) return s;
+  if (!use_decode(plan, CASCADE_BF16, n_heads, n_kv_heads, kHeadDim) || !plan->kv_pos.empty()) {
+    set_error("%s: needs a plan with one query row over the whole cache (cascade_shard_plan with n_q = 1) and "
+              "n_heads / n_kv_heads in {1,2,4,8}", fn);
+    return CASCADE_ERR_UNSUPPORTED;
+  }
+  if (position < 0 || position >= plan->dev.n_kv || position >= n_positions) {
+    set_error("%s: position %d outside the cache of %d rows or the table of %d rows", fn, position, plan->dev.n_kv,
+              n_positions);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(rope_table) || !aligned16(o_out) ||
+      !strides_ok(k_new_strides, 2) || !strides_ok(v_new_strides, 2) || !strides_ok(o_strides, 2)) {
+    set_error("%s: pointers and row strides must be 16-byte aligned", fn);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  const size_t part_bytes = align_up(decode_ws_bytes(plan, CASCADE_BF16, batch, n_heads, kHeadDim), 256);
+  const size_t need = part_bytes + align_up((size_t)batch * n_heads * kHeadDim * 2, 256);
+  if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255)) {
+    set_error("%s: workspace of %zu bytes (256-byte aligned) required, got %zu", fn, need, workspace_bytes);
+    return CASCADE_ERR_WORKSPACE;
+  }
+  // the new token sits at `position`: it is the query position, and the mask admits the cache rows up to it
+  s = cascade_plan_advance(plan, position - plan->q_idx[0], stream);
+  if (s != CASCADE_OK) return s;
+  char* ws = (char*)workspace;
+  void* q_rot = ws + part_bytes;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = launch_append_rope(batch, n_heads, n_kv_heads, q_new, {q_strides.batch, q_strides.token, q_strides.head},
+                                     k_new, {k_new_strides.batch, k_new_strides.token, k_new_strides.head}, v_new,
+                                     {v_new_strides.batch, v_new_strides.token, v_new_strides.head}, q_rot, k_cache,
+                                     {k_cache_strides.batch, k_cache_strides.token, k_cache_strides.head}, v_cache,
+                                     {v_cache_strides.batch, v_cache_strides.token, v_cache_strides.head}, position,
+                                     reinterpret_cast<const float2*>(rope_table), st);
+  if (e != cudaSuccess) return cuda_fail(e, "cascade_decode_step_rope: append launch");
+  const cascade_strides_t qr = {(int64_t)n_heads * kHeadDim, (int64_t)n_heads * kHeadDim, kHeadDim};
+  return attn_sharded_impl(fn, plan, CASCADE_BF16, batch, n_heads, n_kv_heads, kHeadDim, scale, q_rot, qr, k_cache,
+                           k_cache_strides, v_cache, v_cache_strides, nullptr, 0, o_out, o_strides, lse_out, ws, part_bytes,
+                           st);
+}
+
 cascade_status_t cascade_attn_sharded_host(const cascade_plan_t* plan, cascade_dtype_t dtype, int32_t batch,
                                            int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, float scale,
                                            const void* q_host, const void* k_host, const void* v_host, void* o_host,
@@ -934,7 +1036,7 @@ cascade_status_t cascade_attn_sharded_host(const cascade_plan_t* plan, cascade_d
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_sharded_host: cudaGetDevice");
-  if (dev < 0 || dev >= 16) {
+  if (dev < 0 || dev >= 64) {
     set_error("%s: device ordinal %d not supported", fn, dev);
     return CASCADE_ERR_UNSUPPORTED;
   }
@@ -944,12 +1046,17 @@ cascade_status_t cascade_attn_sharded_host(const cascade_plan_t* plan, cascade_d
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&hs.d2h, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&hs.start, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&hs.done, cudaEventDisableTiming);
-    for (int g = 0; g < kMaxHostGroups && e == cudaSuccess; ++g) {
-      e = cudaEventCreateWithFlags(&hs.uploaded[g], cudaEventDisableTiming);
-      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&hs.computed[g], cudaEventDisableTiming);
-    }
     if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_sharded_host: creating streams and events");
     hs.ready = true;
+  }
+  const int n_groups = n_kv_heads / host_call_group(n_heads, n_kv_heads, head_dim, elt_size(dtype));
+  while ((int)hs.uploaded.size() < n_groups) {
+    cudaEvent_t a = nullptr, b = nullptr;
+    e = cudaEventCreateWithFlags(&a, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&b, cudaEventDisableTiming);
+    if (e != cudaSuccess) return cuda_fail(e, "cascade_attn_sharded_host: creating events");
+    hs.uploaded.push_back(a);
+    hs.computed.push_back(b);
   }
   cudaStream_t st = (cudaStream_t)stream;
   char* ws = (char*)workspace;

@@ -102,6 +102,12 @@ cudaError_t launch_attn_simt(const AttnParams& p, cascade_dtype_t dtype, cudaStr
 cudaError_t launch_attn_tc(const AttnParams& p, const void* k_sorted, const void* v_sorted, cudaStream_t stream);
 cudaError_t launch_gather_kv(const AttnParams& p, void* k_out, void* v_out, cudaStream_t stream);
 cudaError_t launch_rope_table(int32_t n_positions, int32_t head_dim, double base, float2* table, cudaStream_t stream);
+cudaError_t launch_rope_apply(cascade_dtype_t dtype, int32_t batch, int32_t n_rows, int32_t n_heads, int32_t head_dim,
+                              const void* x, Strides xs, int32_t first_position, const float2* table, void* y, Strides ys,
+                              cudaStream_t stream);
+cudaError_t launch_append_rope(int32_t batch, int32_t H, int32_t Hkv, const void* q_new, Strides qs, const void* k_new,
+                               Strides kns, const void* v_new, Strides vns, void* q_rot, void* k_cache, Strides kcs,
+                               void* v_cache, Strides vcs, int32_t position, const float2* table, cudaStream_t stream);
 cudaError_t launch_decode(const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_merge(const MergeParams& p, cascade_dtype_t dtype, cudaStream_t stream);
 

@@ -159,3 +159,68 @@ def test_argument_checks(cb, gu):
     for bad in [(0, 128, 10000.0), (8, 127, 10000.0), (8, 128, 1.0)]:
         with pytest.raises(cb.CascadeError):
             cb.cascade_rope_table(*bad)
+
+
+@pytest.mark.parametrize("dtype,d,H", [("bf16", 128, 8), ("bf16", 64, 4), ("f32", 64, 3), ("f32", 128, 2)])
+def test_standalone_rotary_pass_matches_oracle(cb, gu, dtype, d, H):
+    """cascade_rope_apply on a block of rows that starts in the middle of the sequence, out of place and in place, on
+    a strided view."""
+    base, first, n = 10000.0, 37, 45
+    w = wl.make_workload("rope_rows", 2, n, n, H, H, d, dtype, "round_robin", "round_robin", 1, 1, seed=91)
+    (x,) = gu.to_device(w, which=("q",))
+    table = cb.cascade_rope_table(first + n, d, base)
+    want = rope.rotary_pos_emb(w.q, np.arange(first, first + n), base, dtype)
+    y = cb.cascade_rope_apply(x, first, table)
+    packed = torch.cat([x, x], dim=2).contiguous()  # a strided view: heads H..2H-1 of a wider tensor
+    view = packed[:, :, H:]
+    cb.cascade_rope_apply(view, first, table, out=view)
+    torch.cuda.synchronize()
+    for got in (y, view):
+        g = got.double().cpu().numpy()
+        if dtype == "bf16":
+            step = np.maximum(np.abs(want), 2.0 ** -126) * 2.0 ** -7  # one bf16 step at that magnitude
+            assert (np.abs(g - want) <= step).all()
+            assert (g != want).mean() < 5e-3
+        else:
+            assert np.abs(g - want).max() <= 2e-6
+    assert torch.equal(packed[:, :, :H], x)  # the neighbouring heads of the packed tensor are untouched
+
+
+def test_decode_steps_with_rotary_append_over_a_sharded_cache(cb, gu):
+    """A decode loop: every step hands the new token's unrotated q, k, v rows to cascade_decode_step_rope, which appends
+    to a cache whose unwritten rows hold NaN.  Reference: the oracle's rotary step on the whole sequence, then
+    unsharded attention at that position."""
+    base, cap, B, H, Hkv, d, P = 500000.0, 300, 2, 8, 2, 128, 5
+    w = wl.make_workload("decode_rope", B, cap, cap, H, Hkv, d, "bf16", "block_rr", "block_rr", P, P, seed=92, block=4)
+    q_all, k_all, v_all = gu.to_device(w)
+    qr = rope.rotary_pos_emb(w.q, np.arange(cap), base, "bf16").astype(np.float32)
+    kr = rope.rotary_pos_emb(w.k, np.arange(cap), base, "bf16").astype(np.float32)
+    table = cb.cascade_rope_table(cap, d, base)
+    plan = cb.cascade_shard_plan(np.zeros(1, np.int32), w.kv_shard_of, 1, P, 0, True)
+    k_cache = torch.full_like(k_all, float("nan"))
+    v_cache = torch.full_like(v_all, float("nan"))
+    for pos in range(0, 40):
+        o, lse = cb.cascade_decode_step_rope(plan, q_all[:, pos:pos + 1], k_all[:, pos:pos + 1], v_all[:, pos:pos + 1],
+                                             k_cache, v_cache, pos, w.scale, table)
+        o_ref, lse_ref = oracle.attention_unsharded(qr[:, pos:pos + 1], kr, w.v, w.scale, causal=True, q_pos_offset=pos)
+        gu.check_output(o, lse, o_ref, lse_ref, w.tol, f"decode step at position {pos}")
+    # the cache now holds the rotated keys and the values of the tokens seen so far, and nothing else
+    got_k = k_cache[:, :40].double().cpu().numpy()
+    step = np.maximum(np.abs(kr[:, :40]), 2.0 ** -126) * 2.0 ** -7
+    assert (np.abs(got_k - kr[:, :40]) <= step).all()
+    assert torch.equal(v_cache[:, :40], v_all[:, :40]) and torch.isnan(k_cache[:, 40:].float()).all()
+    # jump ahead: fill rows 40..199 in one go with the standalone pass, then continue decoding at position 200
+    cb.cascade_rope_apply(k_all[:, 40:200], 40, table, out=k_cache[:, 40:200])
+    v_cache[:, 40:200] = v_all[:, 40:200]
+    for pos in (200, 201, 299):
+        if pos == 299:
+            cb.cascade_rope_apply(k_all[:, 202:299], 202, table, out=k_cache[:, 202:299])
+            v_cache[:, 202:299] = v_all[:, 202:299]
+        o, lse = cb.cascade_decode_step_rope(plan, q_all[:, pos:pos + 1], k_all[:, pos:pos + 1], v_all[:, pos:pos + 1],
+                                             k_cache, v_cache, pos, w.scale, table)
+        o_ref, lse_ref = oracle.attention_unsharded(qr[:, pos:pos + 1], kr, w.v, w.scale, causal=True, q_pos_offset=pos)
+        gu.check_output(o, lse, o_ref, lse_ref, w.tol, f"decode step at position {pos}")
+    assert plan.device_status() == 0
+    with pytest.raises(cb.CascadeError):
+        cb.cascade_decode_step_rope(plan, q_all[:, :1], k_all[:, :1], v_all[:, :1], k_cache, v_cache, cap, w.scale, table)
+    plan.destroy()
