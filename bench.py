@@ -39,11 +39,13 @@ MIN_STEPS = 20  # timed launches behind every record
 # no capture of the kernel as it stands).  The prefill kernel's traffic grows with batch * KV heads (each (sequence, KV
 # head) streams its own K/V and writes its own output rows), the decode and merge kernels' with the batch.
 NCU_TRAFFIC = {
-    "c2_prefill_8b/attn_tc_kernel": None,
-    "c3_batched/attn_tc_kernel": None,
-    "c4_long_70b/attn_tc_kernel": None,
-    "c5_decode/decode_kernel": None,
-    "c3_batched/merge_kernel": None,
+    "c2_prefill_8b/attn_tc_kernel": (25478656, 1),
+    "c3_batched/attn_tc_kernel": (136032256, 4),        # captured on one of the four sequences
+    "c4_long_70b/attn_tc_kernel": (1212214016, 1),
+    "c3_batched/attn_tc_kernel/partials": (1257771264, 4),
+    "c4_long_70b/attn_tc_kernel/partials": (4671739904, 4),  # captured with a quarter of the heads
+    "c5_decode/decode_kernel": (545430528, 8),          # captured with batch 8 of 64
+    "c3_batched/merge_kernel": (1135894528, 4),
 }
 
 
@@ -240,8 +242,8 @@ def measure_prefill(torch, cb, wl, name, flush, peaks, steps, warmup, seed=None,
     med_p, med_m = statistics.median(ms_p), statistics.median(ms_m)
     rec["partials"] = {"ms": med_p, "tflops": flops / (med_p * 1e-3) / 1e12, "steps": MIN_STEPS,
                        "partial_write_gbs": part_bytes / (kp_ms * 1e-3) / 1e9,
-                       "roofline": _tensor_roofline(peaks, "attn_tc_kernel (one launch over all shard pairs)", flops,
-                                                    kp_ms, kp_n, None)}
+                       "roofline": _tensor_roofline(peaks, "attn_tc_kernel (one CTA per query tile walks all KV shards)",
+                                                    flops, kp_ms, kp_n, _traffic(name + "/attn_tc_kernel/partials"))}
     rec["merge"] = {"ms": med_m, "steps": MIN_STEPS,
                     "roofline": _hbm_roofline(peaks, "merge_kernel", merge_bytes, med_m, MIN_STEPS,
                                               _traffic(name + "/merge_kernel"))}

@@ -311,3 +311,47 @@ def test_scale_must_be_positive_and_finite(gu):
                 call(plan, q, k, v, bad)
             assert ei.value.status == 1
     plan.destroy()
+
+
+@pytest.mark.parametrize("shape", ["tc", "tc_walk_ragged", "decode", "alu"])
+def test_outputs_stay_inside_their_buffers(gu, shape):
+    """Every output buffer is carved out of a larger allocation whose surroundings hold a pattern; after partials,
+    merge and the fused call the pattern must be intact on both sides (the stand-in for a memory checker)."""
+    from paper_2507_05228_b200 import binding as cb
+    w = {"tc": wl.make_workload("canary_tc", 2, 200, 200, 8, 2, 128, "bf16", "random", "random", 3, 3, seed=81),
+         "tc_walk_ragged": wl.make_workload("canary_walk", 1, 333, 333, 4, 1, 128, "bf16", "random", "contiguous", 2, 7,
+                                            seed=82),
+         "decode": wl.make_workload("canary_dec", 3, 1, 500, 8, 2, 128, "bf16", "round_robin", "random", 1, 6, seed=83),
+         "alu": wl.make_workload("canary_alu", 2, 70, 90, 4, 2, 64, "f32", "random", "random", 2, 3, seed=84)}[shape]
+    q, k, v = gu.to_device(w)
+    plan = gu.make_plan(w)
+    pad = 1024  # elements of padding on each side
+
+    def guarded(shape_, dtype, fill):
+        n = int(np.prod(shape_))
+        raw = torch.full((n + 2 * pad,), fill, dtype=dtype, device="cuda")
+        return raw, raw[pad:pad + n].view(shape_)
+
+    B, n_q, H, d, P = w.B, w.n_q, w.H, w.d, w.n_kv_shards
+    bufs = {"o_part": guarded((B, P, n_q, H, d), q.dtype, 7.0), "m_part": guarded((B, P, n_q, H), torch.float32, 7.0),
+            "l_part": guarded((B, P, n_q, H), torch.float32, 7.0), "o": guarded((B, n_q, H, d), q.dtype, 7.0)}
+    code = cb.BF16 if w.dtype == "bf16" else cb.F32
+    ws_bytes = max(cb.cascade_workspace_bytes(plan, cb.CALL_SHARDED, code, B, H, w.Hkv, d),
+                   cb.cascade_workspace_bytes(plan, cb.CALL_PARTIALS, code, B, H, w.Hkv, d), 256)
+    ws_raw = torch.full((ws_bytes + 2 * 4096,), 0x5A, dtype=torch.uint8, device="cuda")
+    off = ((ws_raw.data_ptr() + 2048 + 255) // 256) * 256 - ws_raw.data_ptr()
+    ws = ws_raw[off:off + ws_bytes]
+    parts = (bufs["o_part"][1], bufs["m_part"][1], bufs["l_part"][1])
+    cb.cascade_attn_partials(plan, q, k, v, w.scale, out=parts, workspace=ws)
+    cb.cascade_merge(*parts, plan.dev_ptr("q_idx"), out=bufs["o"][1], want_lse=False)
+    cb.cascade_attn_sharded(plan, q, k, v, w.scale, out=bufs["o"][1], want_lse=False, workspace=ws)
+    torch.cuda.synchronize()
+    for name, (raw, view) in bufs.items():
+        n = view.numel()
+        assert (raw[:pad] == 7.0).all() and (raw[pad + n:] == 7.0).all(), f"{name}: written outside the buffer"
+        assert torch.isfinite(view.float()).all() or name == "m_part"
+    assert (ws_raw[:off] == 0x5A).all() and (ws_raw[off + ws_bytes:] == 0x5A).all(), "workspace overrun"
+    o_ref, _ = oracle.attention_unsharded(w.q, w.k, w.v, w.scale, causal=w.causal, q_pos_offset=w.q_pos_offset)
+    gu.check_output(bufs["o"][1], None, o_ref, None, w.tol, "fused into a guarded buffer")
+    assert plan.device_status() == 0
+    plan.destroy()
