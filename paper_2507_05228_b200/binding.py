@@ -14,7 +14,8 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libcascade_b200.so")
+# CASCADE_B200_LIB selects another build of the same library (the index-checking debug build)
+LIB_PATH = os.environ.get("CASCADE_B200_LIB") or os.path.join(_HERE, "libcascade_b200.so")
 
 F32, BF16 = 0, 1
 CALL_PARTIALS, CALL_SHARDED = 0, 1

@@ -1,4 +1,8 @@
-"""Builds the CUDA library (sm_100a) in-tree with nvcc.  `python -m paper_2507_05228_b200.build [--force]`."""
+"""Builds the CUDA library (sm_100a) in-tree with nvcc.  `python -m paper_2507_05228_b200.build [--force] [--debug]`.
+
+--debug builds libcascade_b200_debug.so with -DCASCADE_DEBUG: every row index a kernel reads out of a plan array is
+checked before it forms an address (a bad one lands in the plan's status word).  Load it by setting the environment
+variable CASCADE_B200_LIB to its path before importing the binding."""
 from __future__ import annotations
 
 import os
@@ -9,6 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcascade_b200.so")
+LIB_DEBUG = os.path.join(HERE, "libcascade_b200_debug.so")
 SOURCES = ["cascade_api.cu", "merge.cu", "attn_simt.cu", "attn_tc.cu", "gather.cu", "decode.cu", "decode_static.cu",
            "shard_maps.cu", "rope.cu"]
 NVCC_FLAGS = [
@@ -24,25 +29,26 @@ def _nvcc() -> str:
     return "nvcc"
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+def _stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "cascade.h"), __file__]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu file for sm_100a and link libcascade_b200.so next to this file."""
-    if not force and not _stale():
-        return LIB
-    objdir = os.path.join(HERE, "_build")
+def build_library(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Compile every .cu file for sm_100a and link libcascade_b200.so (or the _debug variant) next to this file."""
+    lib = LIB_DEBUG if debug else LIB
+    if not force and not _stale(lib):
+        return lib
+    objdir = os.path.join(HERE, "_build_debug" if debug else "_build")
     os.makedirs(objdir, exist_ok=True)
     objs, procs = [], []
     for src in SOURCES:
         obj = os.path.join(objdir, src.replace(".cu", ".o"))
         objs.append(obj)
-        cmd = [_nvcc(), *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
+        cmd = [_nvcc(), *NVCC_FLAGS, *(["-DCASCADE_DEBUG"] if debug else []), "-c", os.path.join(CSRC, src), "-o", obj]
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
     log = []
     failed = False
@@ -56,11 +62,11 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         sys.stderr.write("\n".join(log))
     if failed:
         raise RuntimeError("nvcc failed; see output above")
-    tmp = LIB + f".{os.getpid()}.tmp"
+    tmp = lib + f".{os.getpid()}.tmp"
     subprocess.check_call([_nvcc(), "-shared", "-o", tmp, *objs, "-gencode", "arch=compute_100a,code=sm_100a"])
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

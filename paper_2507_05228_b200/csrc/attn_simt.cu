@@ -66,7 +66,9 @@ __global__ void __launch_bounds__(128) attn_simt_kernel(AttnParams p) {
   // gather the query rows of this tile
   for (int i = tid; i < R * (D / 4); i += 128) {
     const int r = i / (D / 4), c4 = (i % (D / 4)) * 4;
-    if (r < nrows) load_row_chunk<T>(qb + (int64_t)q_idx[row0 + r] * p.qs.token + c4, &sQ[r][c4]);
+    if (r < nrows)
+      load_row_chunk<T>(qb + CASCADE_CHECKED((int64_t)q_idx[row0 + r], pl.n_q, pl.status, 104) * p.qs.token + c4,
+                        &sQ[r][c4]);
     else sQ[r][c4] = sQ[r][c4 + 1] = sQ[r][c4 + 2] = sQ[r][c4 + 3] = 0.f;
   }
 
@@ -91,7 +93,7 @@ __global__ void __launch_bounds__(128) attn_simt_kernel(AttnParams p) {
       for (int i = tid; i < TK * (D / 4); i += 128) {
         const int r = i / (D / 4), c4 = (i % (D / 4)) * 4;
         if (t0 + r < need) {
-          const int64_t tok = kv_idx[base + t0 + r];
+          const int64_t tok = CASCADE_CHECKED((int64_t)kv_idx[base + t0 + r], pl.n_kv, pl.status, 105);
           load_row_chunk<T>(kb + tok * p.ks.token + c4, &sK[r][c4]);
           load_row_chunk<T>(vb + tok * p.vs.token + c4, &sV[r][c4]);
         } else {
@@ -161,7 +163,7 @@ __global__ void __launch_bounds__(128) attn_simt_kernel(AttnParams p) {
     for (int rr = 0; rr < RPW; ++rr) {
       const int r = warp * RPW + rr;
       if (r >= nrows) continue;
-      const int tok = q_idx[row0 + r];
+      const int tok = (int)CASCADE_CHECKED((int64_t)q_idx[row0 + r], pl.n_q, pl.status, 104);
       const float inv = l_run[rr] > 0.f ? 1.f / l_run[rr] : 0.f;
       T* op = static_cast<T*>(p.o_out) + (int64_t)b * p.os.batch + (int64_t)tok * p.os.token +
               (int64_t)h * p.os.head;

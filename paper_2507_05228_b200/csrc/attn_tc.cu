@@ -428,7 +428,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const int r = (tid >> 3 & 15) + 16 * j;
-        const int tok = __ldg(q_idx + sub_row0 + min(r >> lg, sub_nrows - 1));
+        const int tok =
+            (int)CASCADE_CHECKED((int64_t)__ldg(q_idx + sub_row0 + min(r >> lg, sub_nrows - 1)), pl.n_q, pl.status, 108);
         const __nv_bfloat16* row = qb + (int64_t)tok * p.qs.token + (int64_t)(h0 + (r & (Gp - 1))) * p.qs.head;
         qv[2 * j] = __ldg(reinterpret_cast<const uint4*>(row));
         qv[2 * j + 1] = __ldg(reinterpret_cast<const uint4*>(row + 64));
@@ -443,7 +444,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(const __grid_const
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
         const int r = (tid >> 4 & 7) + 8 * j;
-        const int tok = __ldg(q_idx + sub_row0 + min(r >> lg, sub_nrows - 1));
+        const int tok =
+            (int)CASCADE_CHECKED((int64_t)__ldg(q_idx + sub_row0 + min(r >> lg, sub_nrows - 1)), pl.n_q, pl.status, 108);
         qv[j] = __ldg(reinterpret_cast<const uint4*>(qb + (int64_t)tok * p.qs.token +
                                                      (int64_t)(h0 + (r & (Gp - 1))) * p.qs.head));
       }
@@ -787,7 +789,7 @@ if constexpr (kRope) {
       int64_t stat = 0;
       if (row_ok) {
         if (p.fused) {
-          const int tok = __ldg(q_idx + slot);
+          const int tok = (int)CASCADE_CHECKED((int64_t)__ldg(q_idx + slot), pl.n_q, pl.status, 109);
           stat = ((int64_t)b * pl.n_q + tok) * p.H + head;
           dst = static_cast<__nv_bfloat16*>(p.o_out) + (int64_t)b * p.os.batch + (int64_t)tok * p.os.token +
                 (int64_t)head * p.os.head;

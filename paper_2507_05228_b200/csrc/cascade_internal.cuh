@@ -59,6 +59,21 @@ struct AttnParams {
   const float2* rope;
 };
 
+// Debug build (-DCASCADE_DEBUG, libcascade_b200_debug.so): every row index that a kernel reads out of a plan array
+// before it forms an address is checked against the tensor it indexes; a bad one is recorded in the plan's status word
+// (codes 101..; cascade_plan_device_status then fails) and replaced by row 0, so the access itself stays in bounds.
+// The release build compiles the checks away.
+#ifdef CASCADE_DEBUG
+__device__ __forceinline__ int64_t cascade_checked_index(int64_t i, int64_t n, int32_t* status, int code) {
+  if (i >= 0 && i < n) return i;
+  atomicCAS(status, 0, code);
+  return 0;
+}
+#define CASCADE_CHECKED(i, n, status, code) cascade_checked_index((i), (n), (status), (code))
+#else
+#define CASCADE_CHECKED(i, n, status, code) (i)
+#endif
+
 struct MergeParams {
   const void* o_part;
   const float* m_part;

@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(128, 4) decode_kernel(AttnParams p) {
     }
     return;
   }
-  const int tok_q = pl.q_idx[(size_t)map * pl.n_q];
+  const int tok_q = (int)CASCADE_CHECKED((int64_t)pl.q_idx[(size_t)map * pl.n_q], pl.n_q, pl.status, 107);
   const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(p.k) + (int64_t)b * p.ks.batch +
                             (int64_t)g * p.ks.head + 32 * j;
   const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(p.v) + (int64_t)b * p.vs.batch +
@@ -114,13 +114,13 @@ __global__ void __launch_bounds__(128, 4) decode_kernel(AttnParams p) {
     const int last = n_vis - 1;
     // gathered rows: K rows x and x+8 of the block, V rows 2j, 2j+1, 2j+8, 2j+9 (clamped; masked below)
     uint32_t ka[16], kbv[16];
-    load64(kb + (int64_t)__ldg(kv_idx + min(k0 + x, last)) * p.ks.token, ka, 0);
-    load64(kb + (int64_t)__ldg(kv_idx + min(k0 + 8 + x, last)) * p.ks.token, kbv, 0);
+    load64(kb + CASCADE_CHECKED((int64_t)__ldg(kv_idx + min(k0 + x, last)), pl.n_kv, pl.status, 106) * p.ks.token, ka, 0);
+    load64(kb + CASCADE_CHECKED((int64_t)__ldg(kv_idx + min(k0 + 8 + x, last)), pl.n_kv, pl.status, 106) * p.ks.token, kbv, 0);
     uint32_t vr[4][8];
 #pragma unroll
     for (int rr = 0; rr < 4; ++rr) {
       const int key = k0 + 2 * j + (rr & 1) + (rr >> 1) * 8;
-      const uint4* src = reinterpret_cast<const uint4*>(vb + (int64_t)__ldg(kv_idx + min(key, last)) * p.vs.token);
+      const uint4* src = reinterpret_cast<const uint4*>(vb + CASCADE_CHECKED((int64_t)__ldg(kv_idx + min(key, last)), pl.n_kv, pl.status, 106) * p.vs.token);
       const uint4 t0 = __ldcs(src), t1 = __ldcs(src + 1);
       vr[rr][0] = t0.x; vr[rr][1] = t0.y; vr[rr][2] = t0.z; vr[rr][3] = t0.w;
       vr[rr][4] = t1.x; vr[rr][5] = t1.y; vr[rr][6] = t1.z; vr[rr][7] = t1.w;

@@ -19,8 +19,9 @@ constexpr int kGatherRowsPerCta = 64;
 // prefix seen by the query row with the largest position (the last token of the query block).
 __device__ __forceinline__ bool slot_is_visible(const PlanDev& pl, int map, int slot) {
   const int P = pl.n_kv_shards;
-  const int kk = __ldg(pl.kv_slot_shard + (size_t)map * pl.n_kv + slot);
-  const int last_slot = __ldg(pl.q_inv + (size_t)map * pl.n_q + pl.n_q - 1);
+  const int kk = (int)CASCADE_CHECKED((int64_t)__ldg(pl.kv_slot_shard + (size_t)map * pl.n_kv + slot), P, pl.status, 102);
+  const int last_slot =
+      (int)CASCADE_CHECKED((int64_t)__ldg(pl.q_inv + (size_t)map * pl.n_q + pl.n_q - 1), pl.n_q, pl.status, 103);
   const int longest = __ldg(pl.vis + ((size_t)map * pl.n_q + last_slot) * P + kk);
   return slot - __ldg(pl.kv_off + (size_t)map * (P + 1) + kk) < longest;
 }
@@ -45,7 +46,7 @@ __global__ void __launch_bounds__(256) gather_kv_kernel(AttnParams p, __nv_bfloa
     const int slot = slot0 + 16 * i + r0;
     kr[i] = vr[i] = make_uint4(0u, 0u, 0u, 0u);
     if (slot < pl.n_kv && slot_is_visible(pl, map, slot)) {
-      const int64_t tok = __ldg(kv_idx + slot);
+      const int64_t tok = CASCADE_CHECKED((int64_t)__ldg(kv_idx + slot), pl.n_kv, pl.status, 101);
       kr[i] = __ldcs(reinterpret_cast<const uint4*>(kb + tok * p.ks.token + chunk * 8));
       vr[i] = __ldcs(reinterpret_cast<const uint4*>(vb + tok * p.vs.token + chunk * 8));
     }
@@ -100,7 +101,7 @@ __global__ void __launch_bounds__(256) gather_kv_rope_kernel(AttnParams p, __nv_
     klo[i] = khi[i] = vlo[i] = vhi[i] = make_uint4(0u, 0u, 0u, 0u);
     tok[i] = -1;
     if (slot < pl.n_kv && slot_is_visible(pl, map, slot)) {
-      tok[i] = __ldg(kv_idx + slot);
+      tok[i] = (int)CASCADE_CHECKED((int64_t)__ldg(kv_idx + slot), pl.n_kv, pl.status, 101);
       const __nv_bfloat16* kr = kb + (int64_t)tok[i] * p.ks.token + chunk * 8;
       const __nv_bfloat16* vr = vb + (int64_t)tok[i] * p.vs.token + chunk * 8;
       klo[i] = __ldcs(reinterpret_cast<const uint4*>(kr));
