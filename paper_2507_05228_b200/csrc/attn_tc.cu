@@ -6,8 +6,11 @@
 // are spread over the whole sequence, and the staircase between the shortest and the longest visible prefix of a
 // tile is wasted tensor work; stacking heads shrinks that staircase by Gp.
 // One CTA owns two such sub-tiles (the next 128 / Gp slots of the same shard, same heads), which share every K/V
-// tile, and either one KV shard (partials: the Attention-Pass algorithm for the pair) or all KV shards one after another (fused:
-// the carry n, w, o of the Post-Pass algorithm is the running max / sum / output of the streaming softmax).
+// tile, and walks all KV shards one after another.  Fused route: the carry n, w, o of the Post-Pass algorithm is the
+// running max / sum / output of the streaming softmax, and one output row is written at the end.  Partials (kWalk,
+// the Attention-Pass algorithm for every pair of the query tile): a tile never mixes two shards, and at every shard
+// boundary that shard's (u, m, l) is written out and the statistics and the accumulator start over.  (A CTA per
+// (query tile, KV shard) pair is kept as a compile-time alternative; it pays the CTA set-up once per pair.)
 // The KV shards are walked one after another; each shard's visible prefix (as seen by the CTA's last row, which has
 // the longest one) is cut into chunks of 32 keys, and four consecutive chunks of that stream - possibly from
 // different shards - form one MMA tile of 128 keys, so that only the last tile of a CTA is narrower.  (An MMA costs
