@@ -342,12 +342,21 @@ def measure_exchange(torch, cb, cd, wl, flush, rank, world):
 
     ms = _time_steps(torch, step, MIN_STEPS, 3, flush)
     total_ms = cd.max_over_ranks(sum(ms)) / MIN_STEPS
+    direct_ms = None
+    if world == 1:
+        # the one-kernel form of stage B + post-pass (cascade_merge_peers reads the parts where they were written);
+        # with several ranks the sources would be the peers' buffers mapped into this process, which is not wired here
+        def step_direct():
+            ra.combine_in_place([ra.partials(q, k_res, v_res, w.scale)], want_lse=True)
+
+        direct_ms = statistics.median(_time_steps(torch, step_direct, MIN_STEPS, 3, flush))
     wire = cd.sum_over_ranks(float(sent[0]))
     rec = {"workload": "one 8B-shaped sequence of 8192 tokens, 16 x 16 random shards, KV shards dealt round-robin to "
                        "the ranks", "world": world, "ms_per_layer": total_ms, "steps": MIN_STEPS,
            "tflops": w.flops() / (total_ms * 1e-3) / 1e12, "stage_b_bytes_sent": wire,
            "stage_b_bytes_closed_form": ex.stage_b_bytes(w.B, w.n_kv_shards, w.n_q, w.H, w.d, 2),
            "wire": "nccl all_to_all_single" if world > 1 else "none (one rank: local copy)",
+           "ms_per_layer_parts_read_in_place": direct_ms,
            "device_status": ra.plan.device_status()}
     ra.destroy()
     return rec

@@ -210,6 +210,30 @@ cascade_status_t cascade_merge(cascade_dtype_t dtype, int32_t batch, int32_t n_p
                                float* lse_out, void* stream);
 
 /*
+ * cascade_merge_peers -- stage B of the layer and the post-pass combine in one kernel (Single Layer Forward Pass
+ * algorithm: "CompNode_i gets m, e, u" from the AttnNodes, then the Post-Pass algorithm; Section 5.2.3): the parts are
+ * read where they were computed instead of being copied to the combining party first.  Source s is the set of
+ * partial buffers one party wrote with cascade_attn_partials for ITS KV shards (cascade_shard_plan_resident):
+ *   o_parts[s]  DEVICE [batch][parts_per_source[s]][n_source_rows][n_heads][head_dim] in `dtype`
+ *   m_parts[s], l_parts[s]  DEVICE fp32 [batch][parts_per_source[s]][n_source_rows][n_heads]
+ * The three pointer tables and parts_per_source are HOST arrays of n_sources entries (at most 16).  A source pointer
+ * may address another GPU's memory that is mapped into this process (CUDA IPC, peer access): the kernel reads it
+ * with plain loads, each 16-byte piece once; it uses no multicast and no TMA.  The caller orders this call after the
+ * writers of every source (their streams, or a barrier between processes).
+ *   row_gather  DEVICE int32 [n_rows] or NULL: the row of the source buffers (shard-major slot of the whole sequence)
+ *               that output row r combines -- the rows of the query shards this party owns; NULL = row r
+ *   o_out       [batch][n_rows][n_heads][head_dim] with strides;  lse_out optional fp32 [batch][n_rows][n_heads]
+ * The result equals cascade_merge over the union of all sources' parts restricted to the gathered rows.
+ * Errors: INVALID_ARG, UNSUPPORTED (dtype, head_dim, more than 16 sources), CUDA.
+ */
+cascade_status_t cascade_merge_peers(cascade_dtype_t dtype, int32_t batch, int32_t n_sources,
+                                     const void* const* o_parts, const float* const* m_parts,
+                                     const float* const* l_parts, const int32_t* parts_per_source,
+                                     int32_t n_source_rows, const int32_t* row_gather, int32_t n_rows,
+                                     int32_t n_heads, int32_t head_dim, void* o_out, cascade_strides_t o_strides,
+                                     float* lse_out, void* stream);
+
+/*
  * cascade_attn_sharded -- attention-pass and post-pass fused (the Attention-Pass algorithm followed by the Post-Pass algorithm): walks the KV shards of the plan one after another for each query-shard tile and carries
  * (n, w, o) across shards, so no partial is written to memory; by the identity of Section 5.2.3 the
  * result equals cascade_merge(cascade_attn_partials(...)).  Output in token order:

@@ -33,7 +33,7 @@ EXPORTS = [
     "cascade_kernel_timing_begin", "cascade_kernel_timing_end", "cascade_rope_table", "cascade_attn_sharded_rope",
     "cascade_cdelta_shard_map", "cascade_msplit_shard_map", "cascade_index_set_gaps", "cascade_kl_gaps",
     "cascade_attn_sharded_host", "cascade_plan_advance", "cascade_shard_plan_resident",
-    "cascade_shard_plan_resident_host", "cascade_rope_apply", "cascade_decode_step_rope",
+    "cascade_shard_plan_resident_host", "cascade_rope_apply", "cascade_decode_step_rope", "cascade_merge_peers",
 ]
 
 
@@ -70,6 +70,7 @@ def lib() -> ctypes.CDLL:
         L.cascade_rope_apply.argtypes = [i32, i32, i32, i32, i32, vp, Strides, i32, vp, i32, vp, Strides, vp]
         L.cascade_decode_step_rope.argtypes = [vp, i32, i32, i32, f32, vp, Strides, vp, Strides, vp, Strides, vp, Strides,
                                                vp, Strides, i32, vp, i32, vp, Strides, vp, vp, ctypes.c_size_t, vp]
+        L.cascade_merge_peers.argtypes = [i32, i32, i32, vp, vp, vp, vp, i32, vp, i32, i32, i32, vp, Strides, vp, vp]
         L.cascade_plan_destroy.argtypes = [vp]
         L.cascade_plan_get.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(i64)]
         L.cascade_plan_dense_mask.argtypes = [vp, i32, i32, i32, vp, i64]
@@ -301,6 +302,27 @@ def cascade_merge(o_part: torch.Tensor, m_part: torch.Tensor, l_part: torch.Tens
     _check(lib().cascade_merge(code, B, P, n_rows, H, d, o_part.data_ptr(), m_part.data_ptr(), l_part.data_ptr(),
                                row_scatter_ptr or None, row_scatter_batch_stride, o.data_ptr(), _strides(o),
                                lse.data_ptr() if lse is not None else None, _stream()))
+    return o, lse
+
+
+def cascade_merge_peers(sources, row_gather: Optional[torch.Tensor], n_rows: int, out=None, want_lse: bool = True):
+    """Post-pass over parts left where they were computed.  sources: list of (o_part [B, P_s, n_src_rows, H, d],
+    m_part, l_part [B, P_s, n_src_rows, H]) device tensors, one triple per party (P_s may differ); row_gather: device
+    int32 [n_rows] rows of the source buffers to combine, or None.  Returns (o [B, n_rows, H, d], lse or None)."""
+    o0 = sources[0][0]
+    B, _, n_src_rows, H, d = o0.shape
+    n = len(sources)
+    VP = ctypes.c_void_p * n
+    ptr = lambda t: t.data_ptr() if t.numel() else None
+    o_ptrs = VP(*[ptr(s[0]) for s in sources])
+    m_ptrs = VP(*[ptr(s[1]) for s in sources])
+    l_ptrs = VP(*[ptr(s[2]) for s in sources])
+    parts = (ctypes.c_int32 * n)(*[s[0].shape[1] for s in sources])
+    o = out if out is not None else torch.empty((B, n_rows, H, d), dtype=o0.dtype, device=o0.device)
+    lse = torch.empty((B, n_rows, H), dtype=torch.float32, device=o0.device) if want_lse else None
+    _check(lib().cascade_merge_peers(_dtype_code(o0), B, n, o_ptrs, m_ptrs, l_ptrs, parts, n_src_rows,
+                                     row_gather.data_ptr() if row_gather is not None else None, n_rows, H, d,
+                                     o.data_ptr(), _strides(o), lse.data_ptr() if lse is not None else None, _stream()))
     return o, lse
 
 

@@ -771,6 +771,71 @@ cascade_status_t cascade_merge(cascade_dtype_t dtype, int32_t batch, int32_t n_p
   return CASCADE_OK;
 }
 
+cascade_status_t cascade_merge_peers(cascade_dtype_t dtype, int32_t batch, int32_t n_sources,
+                                     const void* const* o_parts, const float* const* m_parts,
+                                     const float* const* l_parts, const int32_t* parts_per_source,
+                                     int32_t n_source_rows, const int32_t* row_gather, int32_t n_rows,
+                                     int32_t n_heads, int32_t head_dim, void* o_out, cascade_strides_t o_strides,
+                                     float* lse_out, void* stream) {
+  const char* fn = "cascade_merge_peers";
+  if (!o_parts || !m_parts || !l_parts || !parts_per_source || !o_out) {
+    set_error("%s: null pointer", fn);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (dtype != CASCADE_F32 && dtype != CASCADE_BF16) {
+    set_error("%s: unknown dtype %d", fn, (int)dtype);
+    return CASCADE_ERR_UNSUPPORTED;
+  }
+  if (n_sources < 1 || n_sources > kMaxMergeSources) {
+    set_error("%s: between 1 and %d sources", fn, kMaxMergeSources);
+    return CASCADE_ERR_UNSUPPORTED;
+  }
+  if (batch < 1 || n_source_rows < 1 || n_rows < 1 || n_heads < 1) {
+    set_error("%s: sizes must be positive", fn);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  if (head_dim != 64 && head_dim != 128) {
+    set_error("%s: head_dim %d unsupported (64 or 128)", fn, head_dim);
+    return CASCADE_ERR_UNSUPPORTED;
+  }
+  if (!aligned16(o_out) || !strides_ok(o_strides, elt_size(dtype))) {
+    set_error("%s: output pointer and row strides must be 16-byte aligned", fn);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  MergePeersParams p;
+  memset(&p, 0, sizeof(p));
+  int total_parts = 0;
+  for (int s = 0; s < n_sources; ++s) {
+    if (parts_per_source[s] < 0 || (parts_per_source[s] > 0 && (!o_parts[s] || !m_parts[s] || !l_parts[s])) ||
+        !aligned16(o_parts[s])) {
+      set_error("%s: source %d: null or misaligned buffer, or a negative part count", fn, s);
+      return CASCADE_ERR_INVALID_ARG;
+    }
+    p.o_src[s] = o_parts[s];
+    p.m_src[s] = m_parts[s];
+    p.l_src[s] = l_parts[s];
+    p.parts[s] = parts_per_source[s];
+    total_parts += parts_per_source[s];
+  }
+  if (total_parts < 1) {
+    set_error("%s: no parts", fn);
+    return CASCADE_ERR_INVALID_ARG;
+  }
+  p.n_src = n_sources;
+  p.n_src_rows = n_source_rows;
+  p.row_gather = row_gather;
+  p.o_out = o_out;
+  p.os = {o_strides.batch, o_strides.token, o_strides.head};
+  p.lse_out = lse_out;
+  p.batch = batch;
+  p.n_rows = n_rows;
+  p.H = n_heads;
+  p.d = head_dim;
+  cudaError_t e = launch_merge_peers(p, dtype, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e, "cascade_merge_peers: launch");
+  return CASCADE_OK;
+}
+
 }  // extern "C"
 
 // The fused route; rope_table != null adds the rotary step (cascade_attn_sharded_rope).

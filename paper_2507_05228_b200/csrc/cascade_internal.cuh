@@ -86,6 +86,21 @@ struct MergeParams {
   int32_t batch, n_parts, n_rows, H, d;
 };
 
+// Post-pass that reads every part from the buffer of the party that computed it (cascade_merge_peers).
+constexpr int kMaxMergeSources = 16;
+struct MergePeersParams {
+  const void* o_src[kMaxMergeSources];   // source s: [batch][parts[s]][n_src_rows][H][d]
+  const float* m_src[kMaxMergeSources];  //           [batch][parts[s]][n_src_rows][H]
+  const float* l_src[kMaxMergeSources];
+  int32_t parts[kMaxMergeSources];
+  int32_t n_src, n_src_rows;
+  const int32_t* row_gather;  // [n_rows]: row of the source buffers that output row r combines; null = r
+  void* o_out;
+  Strides os;
+  float* lse_out;
+  int32_t batch, n_rows, H, d;
+};
+
 }  // namespace cascade
 
 struct cascade_plan {
@@ -125,5 +140,6 @@ cudaError_t launch_append_rope(int32_t batch, int32_t H, int32_t Hkv, const void
                                void* v_cache, Strides vcs, int32_t position, const float2* table, cudaStream_t stream);
 cudaError_t launch_decode(const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_merge(const MergeParams& p, cascade_dtype_t dtype, cudaStream_t stream);
+cudaError_t launch_merge_peers(const MergePeersParams& p, cascade_dtype_t dtype, cudaStream_t stream);
 
 }  // namespace cascade

@@ -121,6 +121,101 @@ __global__ void __launch_bounds__(256, 8) merge_kernel(MergeParams p) {
     p.lse_out[((int64_t)b * p.n_rows + out_row) * p.H + h] = w > 0.f ? n + logf(w) : -INFINITY;
 }
 
+// The same combine with the parts left where they were computed: source s (a party's partial buffers, possibly in
+// another GPU's memory mapped into this process) holds parts[s] parts of every row; output row r combines row
+// row_gather[r] of every source.  Stage B of the layer and the post-pass in one kernel: each 16-byte piece of a part
+// crosses the link once, straight into the registers that accumulate it, with plain loads (no staging copy, no
+// multicast).  Same thread mapping as merge_kernel.
+template <typename T, int D>
+__global__ void __launch_bounds__(256, 8) merge_peers_kernel(const __grid_constant__ MergePeersParams p) {
+  using VT = Vec16<T>;
+  constexpr int V = VT::N;
+  constexpr int TPR = D / V;
+  constexpr int ITEMS = 256 / TPR;
+  constexpr int CH = 2;
+  const int sub = threadIdx.x % TPR;
+  const int lane = threadIdx.x & 31;
+  const int group_lane0 = lane - sub;
+  const int64_t per_batch = (int64_t)p.n_rows * p.H;
+  const int64_t total = per_batch * p.batch;
+  int64_t item = (int64_t)blockIdx.x * ITEMS + threadIdx.x / TPR;
+  const bool active = item < total;
+  if (!active) item = total - 1;
+  const int b = (int)(item / per_batch);
+  const int64_t rh = item - (int64_t)b * per_batch;
+  const int r = (int)(rh / p.H);
+  const int h = (int)(rh - (int64_t)r * p.H);
+  const int src_row = p.row_gather ? __ldg(p.row_gather + r) : r;
+  const int64_t part_stride = (int64_t)p.n_src_rows * p.H;       // elements of m / l between two parts of a source
+  const int64_t row_off = (int64_t)src_row * p.H + h;
+
+  float n = -INFINITY;
+  for (int s = 0; s < p.n_src; ++s) {
+    const float* mp = p.m_src[s] + (int64_t)b * p.parts[s] * part_stride + row_off;
+    for (int k = sub; k < p.parts[s]; k += TPR) n = fmaxf(n, __ldg(mp + (int64_t)k * part_stride));
+  }
+#pragma unroll
+  for (int off = TPR / 2; off > 0; off >>= 1) n = fmaxf(n, __shfl_xor_sync(0xffffffffu, n, off));
+
+  float acc[V];
+#pragma unroll
+  for (int i = 0; i < V; ++i) acc[i] = 0.f;
+  float w = 0.f;
+  for (int s = 0; s < p.n_src; ++s) {
+    const int P = p.parts[s];
+    const float* mp = p.m_src[s] + (int64_t)b * P * part_stride + row_off;
+    const float* lp = p.l_src[s] + (int64_t)b * P * part_stride + row_off;
+    const T* up = static_cast<const T*>(p.o_src[s]) + ((int64_t)b * P * part_stride + row_off) * D + sub * V;
+    for (int base = 0; base < P; base += TPR) {
+      float wt = 0.f;
+      if (base + sub < P) {
+        const float mk = __ldg(mp + (int64_t)(base + sub) * part_stride);
+        const float lk = __ldg(lp + (int64_t)(base + sub) * part_stride);
+        wt = lk > 0.f ? expf(mk - n) * lk : 0.f;
+      }
+      w += wt;
+      const int cnt = min(TPR, P - base);  // warp-uniform
+      for (int c0 = 0; c0 < cnt; c0 += CH) {
+        typename VT::Raw u[CH];
+#pragma unroll
+        for (int c = 0; c < CH; ++c)
+          if (c0 + c < cnt) u[c] = VT::load(up + (int64_t)(base + c0 + c) * part_stride * D);
+#pragma unroll
+        for (int c = 0; c < CH; ++c)
+          if (c0 + c < cnt) {
+            const float wc = __shfl_sync(0xffffffffu, wt, group_lane0 + c0 + c);
+            VT::fma(acc, u[c], wc);
+          }
+      }
+    }
+  }
+#pragma unroll
+  for (int off = TPR / 2; off > 0; off >>= 1) w += __shfl_xor_sync(0xffffffffu, w, off);
+  if (!active) return;
+  const float inv = w > 0.f ? 1.f / w : 0.f;
+#pragma unroll
+  for (int i = 0; i < V; ++i) acc[i] *= inv;
+  T* op = static_cast<T*>(p.o_out) + (int64_t)b * p.os.batch + (int64_t)r * p.os.token + (int64_t)h * p.os.head + sub * V;
+  VT::store(op, acc);
+  if (p.lse_out && sub == 0) p.lse_out[((int64_t)b * p.n_rows + r) * p.H + h] = w > 0.f ? n + logf(w) : -INFINITY;
+}
+
+cudaError_t launch_merge_peers(const MergePeersParams& p, cascade_dtype_t dtype, cudaStream_t stream) {
+  const int64_t items = (int64_t)p.batch * p.n_rows * p.H;
+  auto go = [&](auto kern, int items_per_cta) {
+    const int64_t grid = (items + items_per_cta - 1) / items_per_cta;
+    kern<<<(unsigned)grid, 256, 0, stream>>>(p);
+    count_launch();
+    return cudaGetLastError();
+  };
+  if (dtype == CASCADE_BF16) {
+    if (p.d == 128) return go(merge_peers_kernel<__nv_bfloat16, 128>, 256 / 16);
+    return go(merge_peers_kernel<__nv_bfloat16, 64>, 256 / 8);
+  }
+  if (p.d == 128) return go(merge_peers_kernel<float, 128>, 256 / 32);
+  return go(merge_peers_kernel<float, 64>, 256 / 16);
+}
+
 cudaError_t launch_merge(const MergeParams& p, cascade_dtype_t dtype, cudaStream_t stream) {
   const int64_t items = (int64_t)p.batch * p.n_rows * p.H;
   auto go = [&](auto kern, int items_per_cta) {

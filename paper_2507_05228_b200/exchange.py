@@ -172,6 +172,7 @@ class RankAttention:
         q_idx = self.plan.get("q_idx")[0].reshape(-1)
         self.owned_tokens = q_idx[self.stage.my_slots]  # output row r of ``run`` is this token
         self.parts = None
+        self._gather = None
 
     def partials(self, q: torch.Tensor, k_res: torch.Tensor, v_res: torch.Tensor, scale: float, workspace=None):
         self.parts = self.cb.cascade_attn_partials(self.plan, q, k_res, v_res, scale, out=self.parts,
@@ -185,6 +186,18 @@ class RankAttention:
             B, _, _, H, d = u.shape
             return u.new_empty((B, 0, H, d)), (m.new_empty((B, 0, H)) if want_lse else None)
         return self.cb.cascade_merge(u, m, l, 0, want_lse=want_lse)
+
+    def combine_in_place(self, sources, want_lse: bool = True):
+        """Stage B and the post-pass in one kernel (``cascade_merge_peers``): ``sources[s]`` are the partial buffers
+        (o_part, m_part, l_part) of rank s, left where rank s wrote them and reachable from this GPU - the rank's own
+        tensors, or a peer's buffers mapped into this process.  No packing, no all-to-all, no staging copy: the kernel
+        gathers this rank's rows from every source with plain loads.  Rows in the order of ``owned_tokens``."""
+        if self.stage.my_slots.size == 0:
+            B, _, _, H, d = sources[0][0].shape
+            return sources[0][0].new_empty((B, 0, H, d)), None
+        if self._gather is None:
+            self._gather = torch.from_numpy(self.stage.my_slots.astype(np.int32)).to(sources[0][0].device)
+        return self.cb.cascade_merge_peers(sources, self._gather, self.stage.my_slots.size, want_lse=want_lse)
 
     def run(self, q, k_res, v_res, scale, group=None, workspace=None):
         """partials -> stage-B all-to-all -> post-pass.  Returns (o [B, owned rows, H, d], lse, bytes_sent)."""

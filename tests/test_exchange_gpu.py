@@ -42,10 +42,18 @@ def _run_ranks(gu, w, world):
     es = 2 if w.dtype == "bf16" else 4
     assert sent == ex.stage_b_bytes(w.B, w.n_kv_shards, w.n_q, w.H, w.d, es)
     got = ex.deliver_in_process([ra.stage for ra in ranks], packed, w.B, w.H, w.d)
+    sources = [ra.parts for ra in ranks]  # every rank's partial buffers, left where they were written
     seen = []
     for r, ra in enumerate(ranks):
         o, lse = ra.combine(*got[r])
         rows = ra.owned_tokens
+        # the one-kernel form of stage B + post-pass reads the same parts in place: same arithmetic, same result
+        o_d, lse_d = ra.combine_in_place(sources)
+        assert o_d.shape == o.shape
+        if rows.size:
+            gu.check_output(o_d, lse_d, o_ref[:, rows], lse_ref[:, rows], w.tol, f"{w.name} rank {r}/{world} in place",
+                            stored_partials=True)
+            assert (o_d.float() - o.float()).abs().max().item() <= 2.0 ** -6  # summation order differs at most
         gu.check_output(o, lse, o_ref[:, rows], lse_ref[:, rows], w.tol, f"{w.name} rank {r}/{world} post-pass",
                         stored_partials=True)
         seen.append(rows)

@@ -355,3 +355,44 @@ def test_outputs_stay_inside_their_buffers(gu, shape):
     gu.check_output(bufs["o"][1], None, o_ref, None, w.tol, "fused into a guarded buffer")
     assert plan.device_status() == 0
     plan.destroy()
+
+
+def test_merge_peers_matches_oracle_post_pass_on_split_sources(gu):
+    """cascade_merge_peers on synthetic partials split over three sources with different part counts (one of them
+    empty-handed), gathering a subset of rows in a scrambled order; reference: the oracle's post-pass over all parts."""
+    from paper_2507_05228_b200 import binding as cb
+    rng = np.random.Generator(np.random.PCG64(33))
+    for dtype, d, tol in ((torch.bfloat16, 128, 2e-2), (torch.float32, 64, 1e-4)):
+        B, P, R, H = 2, 7, 41, 3
+        u = rng.standard_normal((B, P, R, H, d)).astype(np.float32)
+        if dtype == torch.bfloat16:
+            u = wl.round_to_bf16(u)
+        m = (rng.standard_normal((B, P, R, H)) * 20).astype(np.float32)
+        l = rng.uniform(1, 30, (B, P, R, H)).astype(np.float32)
+        dead = rng.random((B, P, R, H)) < 0.25
+        dead[1, :, 5, 2] = True  # a row whose parts are all empty
+        m[dead], l[dead] = -np.inf, 0.0
+        u[dead] = 0.0
+        split = [[0, 3, 4], [1, 6], [2, 5]]  # which parts each source holds, in its own order
+        rows = rng.permutation(R)[:17].astype(np.int32)
+        order = [k for s in split for k in s]
+        o_ref, lse_ref = oracle.post_pass(u[:, order][:, :, rows].astype(np.float64), m[:, order][:, :, rows].astype(np.float64),
+                                          l[:, order][:, :, rows].astype(np.float64))
+        sources = [(torch.from_numpy(u[:, s]).cuda().to(dtype).contiguous(), torch.from_numpy(m[:, s]).cuda().contiguous(),
+                    torch.from_numpy(l[:, s]).cuda().contiguous()) for s in split]
+        o, lse = cb.cascade_merge_peers(sources, torch.from_numpy(rows).cuda(), rows.size)
+        gu.check_output(o, lse, o_ref, lse_ref, tol, f"merge_peers {dtype}")
+        where = int(np.flatnonzero(rows == 5)[0]) if (rows == 5).any() else None
+        if where is not None:
+            assert (o[1, where, 2] == 0).all() and torch.isneginf(lse[1, where, 2])
+        # identity gather over all rows == cascade_merge on the concatenated parts
+        o_all, lse_all = cb.cascade_merge_peers(sources, None, R)
+        o_m, lse_m = cb.cascade_merge(torch.from_numpy(u[:, order]).cuda().to(dtype).contiguous(),
+                                      torch.from_numpy(m[:, order]).cuda().contiguous(),
+                                      torch.from_numpy(l[:, order]).cuda().contiguous())
+        # (the two kernels add the parts in different orders: equal up to fp32 summation order, then one rounding)
+        step = 2.0 ** -7 if dtype == torch.bfloat16 else 1e-5
+        assert ((o_all.float() - o_m.float()).abs() <= step * o_m.float().abs().clamp(min=1.0)).all()
+        assert torch.allclose(torch.nan_to_num(lse_all, neginf=-1e30), torch.nan_to_num(lse_m, neginf=-1e30), atol=1e-5)
+    with pytest.raises(cb.CascadeError):
+        cb.cascade_merge_peers(sources * 6, None, R)  # 18 sources: more than the kernel's table holds
