@@ -31,10 +31,8 @@ print("debug build: %%d cases clean" %% len(cases))
 
 
 def test_small_cases_run_clean_on_the_index_checking_build():
-    lib = os.path.join(ROOT, "paper_2507_05228_b200", "libcascade_b200_debug.so")
-    if not os.path.exists(lib):
-        from paper_2507_05228_b200 import build
-        build.build_library(debug=True)
+    from paper_2507_05228_b200 import build
+    lib = build.build_library(debug=True)  # compiles only if the library is missing or older than its sources
     env = dict(os.environ, CASCADE_B200_LIB=lib)
     out = subprocess.run([sys.executable, "-c", CHILD % {"root": ROOT, "tests": os.path.join(ROOT, "tests")}], env=env,
                          capture_output=True, text=True, timeout=900)
