@@ -56,6 +56,17 @@ def stage_b_bytes(batch: int, n_kv_shards: int, n_q: int, n_heads: int, head_dim
     return batch * n_kv_shards * n_q * n_heads * (head_dim * u_elt_bytes + 8)
 
 
+def stage_a_elements(batch: int, beta: int, n_tokens: int, n_heads: int, n_kv_heads: int, head_dim: int) -> int:
+    """Closed form of the stage-A payload (sharded q, k, v rows to the AttnNodes): beta d (H + 2 H_KV) N elements."""
+    return batch * beta * head_dim * (n_heads + 2 * n_kv_heads) * n_tokens
+
+
+def layer_comm_bytes(beta: int, elt_bytes: int, head_dim: int, n_heads: int, n_kv_heads: int, n_tokens: int) -> int:
+    """Both stages of one layer: CommBytes = beta F (2 d H + 2 d H_KV + 2 H) N (Section 7.1, "Communication")."""
+    return elt_bytes * (stage_a_elements(1, beta, n_tokens, n_heads, n_kv_heads, head_dim) +
+                        stage_b_elements(1, beta, n_tokens, n_heads, head_dim))
+
+
 class StageB:
     """Routing tables of the stage-B all-to-all for one rank.
 
