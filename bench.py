@@ -425,7 +425,7 @@ def run_ours(args):
         # one KV head group after another with the copies in both directions and the compute overlapped
         cb.cascade_attn_sharded_host(plan, hq, hk, hv, w.scale, ho, ws_host)
 
-    e2e_steps = max(3, min(args.steps, 10))
+    e2e_steps = max(3, min(args.steps, MIN_STEPS))
     ms_e2e = _time_steps(torch, step_e2e, e2e_steps, 3, flush)
     e2e_ms = cd.max_over_ranks(sum(ms_e2e)) / e2e_steps
     h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv))
