@@ -396,3 +396,27 @@ def test_merge_peers_matches_oracle_post_pass_on_split_sources(gu):
         assert torch.allclose(torch.nan_to_num(lse_all, neginf=-1e30), torch.nan_to_num(lse_m, neginf=-1e30), atol=1e-5)
     with pytest.raises(cb.CascadeError):
         cb.cascade_merge_peers(sources * 6, None, R)  # 18 sources: more than the kernel's table holds
+
+
+@pytest.mark.parametrize("seed", [101, 102, 103])
+def test_random_shapes_on_every_route(gu, seed):
+    """Seeded random problems: sizes that are no multiple of any tile, shard counts from 1 to 9 with every map kind,
+    query blocks anywhere in the cache, both masks, several head groupings - every element of plan, partials, merge and
+    fused output against the oracle.  Twelve problems per seed; which route runs follows from the shape."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    kinds = ["random", "contiguous", "round_robin", "block_rr"]
+    heads = [(4, 4), (8, 2), (8, 1), (16, 2), (2, 1), (6, 2)]
+    for trial in range(12):
+        dtype, d = [("bf16", 128), ("bf16", 128), ("bf16", 128), ("f32", 64), ("bf16", 64), ("f32", 128)][trial % 6]
+        H, Hkv = heads[int(rng.integers(len(heads)))]
+        B = int(rng.integers(1, 3))
+        n_q = 1 if trial % 6 == 2 and rng.random() < 0.5 else int(rng.integers(2, 420))
+        n_kv = int(rng.integers(n_q, 640))
+        J = 1 if n_q == 1 else int(rng.integers(1, 7))
+        P = int(rng.integers(1, 10))
+        causal = bool(rng.random() < 0.8)
+        off = n_kv - n_q if rng.random() < 0.6 else int(rng.integers(0, n_kv - n_q + 1))
+        w = wl.make_workload(f"fuzz{seed}_{trial}", B, n_q, n_kv, H, Hkv, d, dtype, kinds[int(rng.integers(4))],
+                             kinds[int(rng.integers(4))], J, P, seed=1000 * seed + trial,
+                             block=int(rng.choice([4, 16, 64])), causal=causal, q_pos_offset=off, symmetric=False)
+        gu.full_parity(w)
