@@ -62,8 +62,12 @@ constexpr int kKStages = 2;  // (a third stage bought nothing)
 constexpr int kVStages = 2;
 constexpr uint32_t kTmemCols = 512;       // S0 | S1 | O0 | O1, 128 columns each; P_s aliases the start of S_s
 constexpr float kRescaleThreshold = 8.f;  // log2 units
+// setmaxnreg only redistributes the registers the CTA was launched with (168 per thread x 384 threads = 64512), and
+// all four warps of an allocation group execute the same instruction: 8 warps x 32 x 216 + 4 warps x 32 x 72 = 64512.
+// An increase that asks for more than the launch grant never returns.
 constexpr int kRegsSoftmax = 216;
 constexpr int kRegsOther = 72;
+static_assert(8 * 32 * kRegsSoftmax + 4 * 32 * kRegsOther <= 168 * kThreads, "setmaxnreg would wait for registers forever");
 constexpr int kChunk = 32;                // keys per chunk of the KV stream
 constexpr int kChunkBytes = kChunk * 128; // one 64-column half of a chunk in a tile
 constexpr int kMaxShards = 256;           // KV shards per CTA whose bookkeeping fits in shared memory
