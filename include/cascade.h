@@ -364,8 +364,11 @@ cascade_status_t cascade_attn_sharded_host(const cascade_plan_t* plan, cascade_d
  * and, for each generated token, writes that token's k and v rows at its index of the caller's cache tensors and
  * calls this function with the token's position: the causal mask (key token <= query position) then admits exactly
  * the cache rows written so far, and the new row belongs to its shard's list without any list being rebuilt.
- * Recomputes VIS and PAIR_CLASS for query position q_pos_offset + token index (host arrays at once, device arrays in
- * stream order); the index lists do not change.  Works for any n_q (a prefill chunk that slides along the sequence);
+ * Recomputes VIS and PAIR_CLASS for query position q_pos_offset + token index; the index lists do not change.  On a
+ * device plan with more than 256 (query row, KV shard) entries two small kernels rewrite the device arrays in stream
+ * order from the plan's own index lists (no host computation, no upload; the host copies that cascade_plan_get and
+ * cascade_plan_dense_mask return are brought up to date when they are next asked for).  Smaller plans (a decode
+ * step), host-only plans and plans over resident K/V rows (kv_pos) recompute on the host and upload in stream order.  Works for any n_q (a prefill chunk that slides along the sequence);
  * the work-sorted order of the plan's query tiles is left as it was built, which affects speed only.
  * Calls that use the plan before and after must be on `stream` or ordered with it.
  * Cache rows beyond the new position need not be initialised (see cascade_attn_partials); rows at or before it must be

@@ -15,7 +15,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcascade_b200.so")
 LIB_DEBUG = os.path.join(HERE, "libcascade_b200_debug.so")
 SOURCES = ["cascade_api.cu", "merge.cu", "attn_simt.cu", "attn_tc.cu", "gather.cu", "decode.cu", "decode_static.cu",
-           "shard_maps.cu", "rope.cu"]
+           "shard_maps.cu", "rope.cu", "plan_advance.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xptxas", "-v", "-I", os.path.join(ROOT, "include"), "-I", CSRC,

@@ -111,6 +111,9 @@ struct cascade_plan {
   std::vector<int4> qtiles[cascade::kNumTileSizes];
   void* dev_blob = nullptr;
   size_t dev_blob_bytes = 0;
+  // cascade_plan_advance moves the device arrays with a kernel; the host copies of vis and pair_class are then brought
+  // up to date only when something reads them (cascade_plan_get, cascade_plan_dense_mask)
+  mutable bool host_vis_stale = false;
 };
 
 namespace cascade {
@@ -139,6 +142,8 @@ cudaError_t launch_append_rope(int32_t batch, int32_t H, int32_t Hkv, const void
                                Strides kns, const void* v_new, Strides vns, void* q_rot, void* k_cache, Strides kcs,
                                void* v_cache, Strides vcs, int32_t position, const float2* table, cudaStream_t stream);
 cudaError_t launch_decode(const AttnParams& p, cudaStream_t stream);
+// vis and pair_class of a device plan recomputed for a new q_pos_offset (plans without kv_pos)
+cudaError_t launch_plan_advance(const PlanDev& d, int32_t q_pos_offset, cudaStream_t stream);
 cudaError_t launch_merge(const MergeParams& p, cascade_dtype_t dtype, cudaStream_t stream);
 cudaError_t launch_merge_peers(const MergePeersParams& p, cascade_dtype_t dtype, cudaStream_t stream);
 

@@ -142,3 +142,19 @@ def sampled_parity(w, per_shard=2, min_rows=0):
     assert plan.device_status() == 0
     plan.destroy()
     return errs, e_merge, e_fused
+
+
+class _DevicePointer:
+    """A raw device pointer presented through the CUDA array interface, so that torch can copy it to the host."""
+
+    def __init__(self, ptr, n, typestr):
+        self.__cuda_array_interface__ = {"shape": (n,), "typestr": typestr, "data": (int(ptr), False), "version": 2}
+
+
+def read_plan_device_array(plan, field):
+    """Device copy of a plan array, fetched with the pointer cascade_plan_get returns (not the library's host copy)."""
+    shape = plan._shape(field)
+    n = int(np.prod(shape))
+    torch.cuda.synchronize()
+    t = torch.as_tensor(_DevicePointer(plan.dev_ptr(field), n, "|u1" if field == "pair_class" else "<i4"), device="cuda")
+    return t.cpu().numpy().reshape(shape)

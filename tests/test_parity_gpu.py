@@ -234,6 +234,38 @@ def test_kernel_timing_counts_attention_launches(gu):
     plan.destroy()
 
 
+def test_plan_advance_on_the_device_matches_a_plan_built_at_that_position(gu):
+    """cascade_plan_advance on a device plan rewrites vis and pair_class with kernels: the device arrays (read through
+    the pointers cascade_plan_get returns), and the host copies refreshed on demand, equal the oracle's plan built for
+    each position, bit for bit; positions before 0 and past the capacity, several maps, a sliding chunk, a
+    bidirectional plan."""
+    from paper_2507_05228_b200 import binding as cb
+    from oracle import sharding
+    n_cap, P = 1000, 7
+    kv_of = np.stack([sharding.cdelta_shard_of(n_cap, 4, 28),
+                      np.random.default_rng(5).integers(0, P, n_cap).astype(np.int32)])
+    q_of = np.zeros((2, 1), np.int32)
+    plan = cb.cascade_shard_plan(q_of, kv_of, 1, P, q_pos_offset=0)
+    for pos in [0, 1, 27, 28, 511, 999, 1000, 5000, -3, 77]:
+        plan.advance(pos)
+        for mp in range(2):
+            ref = oracle.shard_plan(q_of[mp], kv_of[mp], 1, P, q_pos_offset=pos)
+            assert np.array_equal(gu.read_plan_device_array(plan, "vis")[mp], ref.vis), (pos, mp)
+            assert np.array_equal(gu.read_plan_device_array(plan, "pair_class")[mp], ref.pair_class), (pos, mp)
+            assert np.array_equal(plan.get("vis")[mp], ref.vis) and np.array_equal(plan.get("pair_class")[mp], ref.pair_class)
+    plan.destroy()
+    q_chunk = (np.arange(96) % 3).astype(np.int32)
+    for causal in (True, False):
+        plan = cb.cascade_shard_plan(q_chunk, kv_of[0], 3, P, q_pos_offset=0, causal=causal)
+        for off in (0, 96, 500, 904, 950):
+            plan.advance(off)
+            ref = oracle.shard_plan(q_chunk, kv_of[0], 3, P, q_pos_offset=off, causal=causal)
+            assert np.array_equal(gu.read_plan_device_array(plan, "vis")[0], ref.vis), (causal, off)
+            assert np.array_equal(gu.read_plan_device_array(plan, "pair_class")[0], ref.pair_class), (causal, off)
+            assert np.array_equal(plan.dense_mask(1, 2), oracle.dense_mask(ref, 1, 2))
+        plan.destroy()
+
+
 def test_decode_loop_over_a_preallocated_cache_with_plan_advance(gu):
     """Token-sharded KV caching (Appendix F): one plan over the cache capacity, advanced per generated token.  Rows of
     the cache beyond the current position hold arbitrary finite values and must not influence the result."""
