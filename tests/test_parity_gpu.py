@@ -254,15 +254,19 @@ def test_plan_advance_on_the_device_matches_a_plan_built_at_that_position(gu):
             assert np.array_equal(gu.read_plan_device_array(plan, "pair_class")[mp], ref.pair_class), (pos, mp)
             assert np.array_equal(plan.get("vis")[mp], ref.vis) and np.array_equal(plan.get("pair_class")[mp], ref.pair_class)
     plan.destroy()
-    q_chunk = (np.arange(96) % 3).astype(np.int32)
+    # more than 256 (row, shard) entries: the kernels; two maps with different query and KV shardings
+    q_chunk = np.stack([(np.arange(96) % 3), np.random.default_rng(6).integers(0, 3, 96)]).astype(np.int32)
     for causal in (True, False):
-        plan = cb.cascade_shard_plan(q_chunk, kv_of[0], 3, P, q_pos_offset=0, causal=causal)
-        for off in (0, 96, 500, 904, 950):
+        plan = cb.cascade_shard_plan(q_chunk, kv_of, 3, P, q_pos_offset=0, causal=causal)
+        for off in (0, 96, 500, 904, 950, -40):
             plan.advance(off)
-            ref = oracle.shard_plan(q_chunk, kv_of[0], 3, P, q_pos_offset=off, causal=causal)
-            assert np.array_equal(gu.read_plan_device_array(plan, "vis")[0], ref.vis), (causal, off)
-            assert np.array_equal(gu.read_plan_device_array(plan, "pair_class")[0], ref.pair_class), (causal, off)
-            assert np.array_equal(plan.dense_mask(1, 2), oracle.dense_mask(ref, 1, 2))
+            for mp in range(2):
+                ref = oracle.shard_plan(q_chunk[mp], kv_of[mp], 3, P, q_pos_offset=off, causal=causal)
+                assert np.array_equal(gu.read_plan_device_array(plan, "vis")[mp], ref.vis), (causal, off, mp)
+                assert np.array_equal(gu.read_plan_device_array(plan, "pair_class")[mp], ref.pair_class), (causal, off)
+                # the host copies are refreshed by whichever call reads them first
+                assert np.array_equal(plan.dense_mask(1, 2, map=mp), oracle.dense_mask(ref, 1, 2))
+                assert np.array_equal(plan.get("vis")[mp], ref.vis)
         plan.destroy()
 
 
