@@ -46,7 +46,13 @@ def test_unsharded_matches_library_sdpa(causal, H, Hkv, d):
     if causal:
         a = np.where(np.tril(np.ones((37, 37), bool))[None, None], a, -np.inf)
     ref_lse = torch.logsumexp(torch.from_numpy(a), dim=-1).numpy().transpose(0, 2, 1)
-    assert np.abs(lse - ref_lse).max() < 1e-12
+    # The library routine itself wanders: about one process in twenty returns values 1e-9 away from its usual ones (and
+    # from the max-subtracted sum written out below, which the oracle matches to 1e-15 every time), depending on how
+    # the buffer happens to be aligned.  Any mistake in the oracle's statistic would show at 1e-3 or more.
+    assert np.abs(lse - ref_lse).max() < 1e-8
+    m = a.max(-1, keepdims=True)
+    direct = (m[..., 0] + np.log(np.exp(a - m).sum(-1))).transpose(0, 2, 1)
+    assert np.abs(lse - direct).max() < 1e-12
 
 
 def _brute_force(q, k, v, scale, causal, q_pos_offset=0):
@@ -196,7 +202,12 @@ def test_merge_is_stable_and_matches_direct_weighted_average():
     wts = torch.softmax(logw, dim=1).numpy()
     ref = (wts[..., None] * u).sum(1)
     assert np.isfinite(o).all()
-    assert np.abs(o - ref).max() < 1e-12 and np.abs(lse - ref_lse).max() < 1e-10
+    # torch.logsumexp is held to 1e-8 (it is not repeatable below 1e-9, see test_unsharded_matches_library_sdpa);
+    # the same log-space sum written out with numpy is held to 1e-10
+    assert np.abs(o - ref).max() < 1e-12 and np.abs(lse - ref_lse).max() < 1e-8
+    lw = logw.numpy()
+    top = lw.max(1, keepdims=True)
+    assert np.abs(lse - (top[:, 0] + np.log(np.exp(lw - top).sum(1)))).max() < 1e-10
     scatter = np.array([3, 0, 8, 1, 2, 7, 6, 5, 4], np.int32)
     o2, lse2 = oracle.post_pass(u, m, e, row_scatter=scatter)
     assert np.array_equal(o2[:, scatter], o) and np.array_equal(lse2[:, scatter], lse)
